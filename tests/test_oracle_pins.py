@@ -1,0 +1,278 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked without the oracle's own formulas.
+
+Each test names the passage it pins. The brute-force reference here works on unpacked {0,1}
+arrays with bit-by-bit loops, so a mistake in the oracle's packing, popcount, GQA sum,
+tie-break or overwrite shows up as a disagreement.
+"""
+import itertools
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2412_16187_b200 import workloads as wl
+
+
+def unpack(codes, b):
+    """[..., Wd] uint32 -> [..., b] array of 0/1, bit i = column i (LSB first)."""
+    codes = np.asarray(codes, dtype=np.uint32)
+    bits = [(codes[..., i // 32] >> np.uint32(i % 32)) & np.uint32(1) for i in range(b)]
+    return np.stack(bits, axis=-1).astype(np.int64)
+
+
+def pack(bits):
+    bits = np.asarray(bits)
+    b = bits.shape[-1]
+    out = np.zeros(bits.shape[:-1] + ((b + 31) // 32,), dtype=np.uint32)
+    for i in range(b):
+        out[..., i // 32] |= (bits[..., i].astype(np.uint32) << np.uint32(i % 32))
+    return out
+
+
+# ---------------------------------------------------------------- Eq. 2: h(x) = sgn(Rx)
+
+@pytest.mark.parametrize("dtype,d,b", [("f32", 64, 8), ("bf16", 128, 32), ("bf16", 128, 64), ("f32", 40, 24), ("bf16", 128, 16)])
+def test_hash_matches_library_matmul(dtype, d, b):
+    rng = np.random.default_rng(1)
+    W = rng.standard_normal((d, b)).astype(np.float32)
+    x32 = rng.standard_normal((257, d)).astype(np.float32)
+    if dtype == "bf16":
+        x = (x32.view(np.uint32) >> 16).astype(np.uint16)  # truncation is fine: any bf16 pattern is a valid input
+        xd = wl.bf16_to_f32(x).astype(np.float64)
+    else:
+        x, xd = x32, x32.astype(np.float64)
+    codes, fragile, proj = oracle.hash_rows(x, W, dtype, want_fragile=True, want_proj=True)
+    ref = xd @ W.astype(np.float64)  # library routine, fp64
+    np.testing.assert_allclose(proj, ref, rtol=1e-12, atol=1e-12)
+    safe = np.abs(ref) > 1e-9
+    assert np.array_equal(unpack(codes, b)[safe], (ref >= 0).astype(np.int64)[safe])
+    # bits beyond b stay zero
+    if b % 32:
+        assert np.all(codes[:, -1] >> np.uint32(b % 32) == 0)
+    # fragile mask is the stated rule
+    bound = 1e-5 * np.linalg.norm(xd, axis=1)[:, None] * np.linalg.norm(W.astype(np.float64), axis=0)[None, :]
+    assert np.array_equal(unpack(fragile, b), (np.abs(ref) < bound).astype(np.int64))
+
+
+def test_hash_bit_order_and_operand_orientation():
+    # x = e_3 picks row 3 of W; column i of W decides bit i. A transposed W or MSB-first packing fails.
+    d, b = 48, 40
+    W = np.zeros((d, b), dtype=np.float32)
+    on = {0, 1, 5, 31, 32, 39}
+    for i in range(b):
+        W[3, i] = 1.0 if i in on else -1.0
+    W[7, :] = 123.0  # must not matter: x_7 = 0
+    x = np.zeros((1, d), dtype=np.float32)
+    x[0, 3] = 2.5
+    codes = oracle.hash_rows(x, W, "f32")
+    expect = [sum(1 << i for i in on if i < 32), sum(1 << (i - 32) for i in on if i >= 32)]
+    assert codes[0].tolist() == expect
+
+
+def test_hash_sign_conventions():
+    rng = np.random.default_rng(2)
+    d, b = 64, 48
+    W = rng.standard_normal((d, b)).astype(np.float32)
+    x = rng.standard_normal((50, d)).astype(np.float32)
+    c = oracle.hash_rows(x, W, "f32")
+    # scale invariance: h(a x) = h(x) for a > 0 (powers of two keep the products exact)
+    assert np.array_equal(oracle.hash_rows((x * 4.0).astype(np.float32), W, "f32"), c)
+    assert np.array_equal(oracle.hash_rows((x * 0.125).astype(np.float32), W, "f32"), c)
+    # antipodal: every bit flips (no projection is exactly 0 here), so d_H(h(x), h(-x)) = b
+    cneg = oracle.hash_rows(-x, W, "f32")
+    assert np.all((unpack(c, b) ^ unpack(cneg, b)) == 1)
+    # sgn(0) = 1: the zero vector hashes to all ones, -0.0 too
+    z = np.zeros((2, d), dtype=np.float32)
+    z[1] = -0.0
+    cz = oracle.hash_rows(z, W, "f32")
+    assert np.all(unpack(cz, b) == 1) and cz[0].tolist() == [0xFFFFFFFF, 0xFFFF]
+
+
+# ---------------------------------------------------------------- Eq. 3: E[d_H]/b = theta/pi
+
+@pytest.mark.parametrize("theta", [0.0, math.pi / 6, math.pi / 3, math.pi / 2, 2 * math.pi / 3, math.pi])
+def test_simhash_expectation(theta):
+    d, b, trials = 32, 64, 320  # 20480 independent hyperplanes
+    rng = np.random.default_rng(7)
+    x = np.zeros((1, d), dtype=np.float32)
+    y = np.zeros((1, d), dtype=np.float32)
+    x[0, 0] = 1.0
+    y[0, 0], y[0, 1] = math.cos(theta), math.sin(theta)
+    tot = 0
+    for _ in range(trials):
+        W = rng.standard_normal((d, b)).astype(np.float32)
+        tot += int((unpack(oracle.hash_rows(x, W, "f32"), b) ^ unpack(oracle.hash_rows(y, W, "f32"), b)).sum())
+    n = trials * b
+    p = theta / math.pi
+    sigma = math.sqrt(max(p * (1 - p), 1e-12) / n)
+    assert abs(tot / n - p) <= 4 * sigma + 1e-9
+
+
+# ---------------------------------------------------------------- Eq. 5 / Eq. 6 / Algorithm 1: brute force
+
+def brute_victim(table_bits, q_bits, pos, t, n_sink, n_recent):
+    """table_bits [C][b], q_bits [G][b] as 0/1 lists. Returns (victim, distances)."""
+    C = len(table_bits)
+    D = []
+    for j in range(C):
+        dist = 0
+        for g in range(len(q_bits)):
+            for i in range(len(q_bits[g])):
+                if table_bits[j][i] != q_bits[g][i]:
+                    dist += 1
+        D.append(dist)
+    order = [j for j in range(C) if pos[j] >= n_sink and pos[j] < t - n_recent] or list(range(C))
+    worst = max(D[j] for j in order)
+    return min(j for j in order if D[j] == worst), D
+
+
+def make_full_cache(C, b, G, table_codes, n_sink=0, n_recent=0, d=8):
+    oc = oracle.OracleCache(1, 1, G, d, b, C, [C], "f32", n_sink=n_sink, n_recent=n_recent)
+    oc.codes[0, 0] = table_codes
+    oc.pos[0, 0] = np.arange(C)
+    oc.fill[:] = C
+    oc.next_pos[:] = C
+    return oc
+
+
+def test_victim_exhaustive_c3_b3():
+    C, b = 3, 3
+    k = np.ones((1, 1, 8), dtype=np.float32)
+    for table in itertools.product(range(8), repeat=C):
+        for qv in range(8):
+            tb = [[(c >> i) & 1 for i in range(b)] for c in table]
+            qb = [[(qv >> i) & 1 for i in range(b)]]
+            oc = make_full_cache(C, b, 1, np.array(table, dtype=np.uint32).reshape(C, 1))
+            victim, evicted = oc.step_codes(np.array([[[qv]]]), np.array([[[5]]]), k, k)
+            want, D = brute_victim(tb, qb, list(range(C)), C, 0, 0)
+            assert victim[0, 0] == want and evicted[0, 0] == want
+            assert oc.scores[0, 0].tolist() == [-float(x) for x in D]
+            assert oc.codes[0, 0, want, 0] == 5 and oc.pos[0, 0, want] == C
+
+
+@pytest.mark.parametrize("C,b,G", [(8, 8, 1), (8, 8, 2), (5, 40, 2), (7, 64, 4), (6, 33, 3)])
+def test_victim_brute_force_random_tables(C, b, G):
+    rng = np.random.default_rng(C * 100 + b + G)
+    k = np.ones((1, 1, 8), dtype=np.float32)
+    queries = itertools.product(range(256), repeat=G) if b == 8 and G == 1 else None
+    for trial in range(256 if queries is None else 1):
+        tb = rng.integers(0, 2, size=(C, b))
+        # few distinct rows so that ties are common
+        tb[rng.integers(0, C)] = tb[rng.integers(0, C)]
+        qsets = [rng.integers(0, 2, size=(G, b)) for _ in range(4)] if queries is None else \
+            [np.array([[(qv >> i) & 1 for i in range(b)] for qv in qs]) for qs in queries]
+        for qb in qsets:
+            oc = make_full_cache(C, b, G, pack(tb))
+            victim, _ = oc.step_codes(pack(qb)[None], pack(rng.integers(0, 2, size=(1, 1, b))), k, k)
+            want, D = brute_victim(tb.tolist(), qb.tolist(), list(range(C)), C, 0, 0)
+            assert victim[0, 0] == want
+            assert oc.scores[0, 0].tolist() == [-float(x) for x in D]
+
+
+def test_victim_with_protected_tokens():
+    C, b, G = 12, 16, 2
+    rng = np.random.default_rng(11)
+    k = np.ones((1, 1, 8), dtype=np.float32)
+    for trial in range(300):
+        n_sink, n_recent = int(rng.integers(0, 4)), int(rng.integers(0, 4))
+        tb = rng.integers(0, 2, size=(C, b))
+        qb = rng.integers(0, 2, size=(G, b))
+        pos = rng.permutation(40)[:C]
+        t = 40
+        oc = make_full_cache(C, b, G, pack(tb), n_sink=n_sink, n_recent=n_recent)
+        oc.pos[0, 0] = pos
+        oc.next_pos[:] = t
+        victim, evicted = oc.step_codes(pack(qb)[None], pack(rng.integers(0, 2, size=(1, 1, b))), k, k)
+        want, _ = brute_victim(tb.tolist(), qb.tolist(), pos.tolist(), t, n_sink, n_recent)
+        assert victim[0, 0] == want and evicted[0, 0] == pos[want]
+
+
+# ---------------------------------------------------------------- Section 3 state invariants
+
+def run_tiny(n_sink=0, n_recent=0, G=1, b=8, C=16, N=40, T=24, heads=2, d=16, dtype="f32", seed=0):
+    w = wl.Workload("t", seed, 1, 2, heads, G, d, dtype, b, N, C, T, wl.KIND_IID, n_sink=n_sink, n_recent=n_recent)
+    W = wl.gen_W(w)
+    K = wl.gen_tokens(w, "k", 0, 2, 0, N + T)
+    Q = wl.gen_tokens(w, "q", 0, 2, 0, N + T)
+    V = wl.gen_tokens(w, "v", 0, 2, 0, N + T)
+    oc = oracle.OracleCache(2, heads, G, d, b, C, [C, C - 3], dtype, n_sink=n_sink, n_recent=n_recent)
+    return w, W, K, Q, V, oc
+
+
+@pytest.mark.parametrize("n_sink,n_recent,G,b,dtype", [(0, 0, 1, 8, "f32"), (4, 10, 1, 8, "f32"), (2, 3, 4, 40, "bf16"), (0, 5, 2, 64, "bf16")])
+def test_state_invariants_every_step(n_sink, n_recent, G, b, dtype):
+    w, W, K, Q, V, oc = run_tiny(n_sink, n_recent, G, b, dtype=dtype)
+    budgets = oc.budget
+    for t in range(K.shape[2]):
+        q = np.ascontiguousarray(Q[:, :, t])
+        k = np.ascontiguousarray(K[:, :, t])
+        v = np.ascontiguousarray(V[:, :, t])
+        victim, evicted, qc, kc = oc.step(W, q, k, v)
+        for s in range(2):
+            C = int(budgets[s])
+            for h in range(w.n_kv_heads):
+                fill = oc.fill[s, h]
+                assert fill == min(t + 1, C)  # constant budget (Section 3, "Complexity")
+                assert oc.next_pos[s, h] == t + 1
+                slot = victim[s, h]
+                assert oc.pos[s, h, slot] == t  # the newest token is resident (Algorithm 1 lines 3-5)
+                pos = oc.pos[s, h, :fill]
+                assert len(set(pos.tolist())) == fill and np.all(oc.pos[s, h, fill:] == -1)
+                # slot contents belong to the token the slot says it holds; H_t = h(K_t)
+                assert np.array_equal(oc.k_cache[s, h, :fill], K[s, h, pos])
+                assert np.array_equal(oc.v_cache[s, h, :fill], V[s, h, pos])
+                assert np.array_equal(oc.codes[s, h, :fill], oracle.hash_rows(np.ascontiguousarray(K[s, h, pos]), W, dtype))
+                if t + 1 > C:  # protected tokens present once the cache is full and protection is satisfiable
+                    if C > n_sink + n_recent + 1:
+                        present = set(pos.tolist())
+                        assert all(p in present for p in range(min(n_sink, C)))
+                        assert all(p in present for p in range(t - n_recent, t + 1))
+                if t >= C:
+                    assert evicted[s, h] >= 0 and evicted[s, h] not in set(pos.tolist())
+                else:
+                    assert evicted[s, h] == -1 and slot == t
+
+
+def test_prefill_equals_reset_plus_steps_and_short_prompts():
+    w, W, K, Q, V, oc = run_tiny(1, 2, 2, 24, C=16, N=40, T=0, dtype="bf16")
+    plen = np.array([40, 9], dtype=np.int32)  # second prompt is shorter than its budget (13)
+    kc, qc = oc.prefill(W, Q, K, V, plen, want_codes=True)
+    # step-by-step replay, one sequence at a time (sequences are independent)
+    for s in range(2):
+        o1 = oracle.OracleCache(1, w.n_kv_heads, 2, w.head_dim, 24, 16, oc.budget[s:s + 1], "bf16", n_sink=1, n_recent=2)
+        for t in range(int(plen[s])):
+            o1.step(W, np.ascontiguousarray(Q[s:s + 1, :, t]), np.ascontiguousarray(K[s:s + 1, :, t]),
+                    np.ascontiguousarray(V[s:s + 1, :, t]))
+        for name in ("k_cache", "v_cache", "codes", "scores", "pos", "fill", "next_pos"):
+            assert np.array_equal(getattr(o1, name)[0], getattr(oc, name)[s]), name
+    # short prompt: identity placement, nothing evicted
+    assert oc.fill[1].tolist() == [9] * w.n_kv_heads
+    assert np.array_equal(oc.pos[1, :, :9], np.tile(np.arange(9), (w.n_kv_heads, 1)))
+    assert np.array_equal(oc.k_cache[1, :, :9], K[1, :, :9])
+    # prefill on its own codes == prefill from embeddings
+    oc3 = oracle.OracleCache(2, w.n_kv_heads, 2, w.head_dim, 24, 16, oc.budget, "bf16", n_sink=1, n_recent=2)
+    oc3.prefill_codes(kc, qc, K, V, plen)
+    for name in ("k_cache", "v_cache", "codes", "scores", "pos", "fill", "next_pos"):
+        assert np.array_equal(getattr(oc3, name), getattr(oc, name)), name
+
+
+def test_threads_do_not_change_results():
+    w, W, K, Q, V, oc = run_tiny(0, 0, 2, 16)
+    oc.prefill(W, Q, K, V, np.array([64, 64], dtype=np.int32))
+    oc4 = oracle.OracleCache(2, w.n_kv_heads, 2, w.head_dim, 16, 16, oc.budget, "f32", threads=4)
+    oc4.prefill(W, Q, K, V, np.array([64, 64], dtype=np.int32))
+    for name in ("k_cache", "codes", "scores", "pos", "fill"):
+        assert np.array_equal(getattr(oc4, name), getattr(oc, name))
+
+
+# ---------------------------------------------------------------- Section 4.7: hash-table storage
+
+def test_hash_table_storage_closed_form():
+    # Llama-3-70B example: 80 layers, 8 KV heads, sequence 8192, batch 8, 50 % budget -> 80 MB at 32 bits,
+    # i.e. b/8 bytes per slot per KV head. One layer of that shape in the oracle's packed layout:
+    oc = oracle.OracleCache(8, 8, 1, 8, 32, 4096, [4096] * 8, "bf16")
+    assert oc.codes.nbytes * 80 == 80 * 2 ** 20
+    # the paper's 8- and 16-bit figures (20 MB, 40 MB) follow from the same b/8 bytes per slot
+    slots = 80 * 8 * 8 * 4096
+    assert [slots * b // 8 // 2 ** 20 for b in (8, 16, 32)] == [20, 40, 80]
