@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the HashEvict eviction hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One bench step = one pass of the whole hot path over one batch of synthetic input: for every layer replica,
+he_prefill_compress of the prompt batch, then T decode steps, each of which calls he_decode_step once per layer
+replica (layer by layer, as a model would). The decode calls of a step are captured once into a CUDA graph (the
+library neither allocates nor synchronises) and replayed, so the timing is the GPU's, not the Python loop's.
+
+Printed: ONE JSON line. `value` is decode evictions/s (unit-steps per second over all GPUs, inputs resident in
+HBM); prefill keys/s, the roofline fractions, the end-to-end number through the host-buffer entry points and the
+CPU oracle's speed on a bounded sample are further keys of the same line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2412_16187_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode evictions/s (seq x KV-head steps)"
+UNIT = "evictions/s"
+DEFAULT_REPLICAS = {"throughput_batch": 16, "long_prefill": 8, "llama3_8b_gqa": 64, "llama2_7b_layer": 128, "tiny": 4}
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------- bytes
+
+def decode_bytes_per_call(w, budgets, write_scores=True):
+    """Algorithmic bytes one he_decode_step call must move (all units evicting): new q/k/v rows in, codes in,
+    scores out, the victim slot's K/V/code/pos out, victim index out, W once."""
+    d, e, G, b = w.head_dim, w.elem_bytes, w.group_size, w.hash_bits
+    per_unit_fixed = (G + 2) * d * e + 2 * d * e + b / 8 + 8
+    per_slot = b / 8 + (4 if write_scores else 0)
+    slots = float(np.sum(budgets.astype(np.int64))) * w.n_kv_heads
+    return w.n_units * per_unit_fixed + slots * per_slot + d * b * 4
+
+
+def prefill_bytes_per_call(w, budgets, plens):
+    """Algorithmic bytes of one he_prefill_compress call: K hashed once, Q rows of evicting tokens hashed once,
+    surviving K/V read and written once, code/pos/score tables written."""
+    d, e, G, b, H = w.head_dim, w.elem_bytes, w.group_size, w.hash_bits, w.n_kv_heads
+    N = plens.astype(np.int64)
+    C = np.minimum(budgets.astype(np.int64), N)
+    per_seq = N * d * e + (N - C) * G * d * e + 2 * C * d * e + 2 * C * d * e + C * (b / 8 + 8)
+    return float(per_seq.sum()) * H
+
+
+# ------------------------------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        fd, self.path = tempfile.mkstemp(suffix=".csv")
+        os.close(fd)
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [r.split(", ") for r in open(self.path).read().strip().splitlines() if r.count(",") >= 6]
+        os.unlink(self.path)
+        if not rows:
+            return out
+        sm = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].strip() == "Active" for r in rows)]
+        out.update(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=float(rows[0][1]), reasons=reasons,
+                   samples=len(rows), power_w_max=max(float(r[2]) for r in rows))
+        return out
+
+
+# ------------------------------------------------------------------------------------------------- oracle legs
+
+def oracle_sample(w, seqs, decode_steps, threads):
+    """Times the CPU oracle, as it stands, on the first `seqs` sequences: prefill then `decode_steps` steps."""
+    import oracle
+
+    ws = w.scaled(batch=seqs, layers=1)
+    budgets, plens = w.budgets()[:seqs], w.prompt_lens()[:seqs]
+    Nmax = int(plens.max())
+    W = wl.gen_W(w)
+    K = np.zeros((seqs, w.n_kv_heads, Nmax, w.head_dim), dtype=wl.np_dtype(w))
+    V = np.zeros_like(K)
+    Q = np.zeros((seqs, w.n_kv_heads * w.group_size, Nmax, w.head_dim), dtype=wl.np_dtype(w))
+    for s in range(seqs):
+        n = int(plens[s])
+        K[s, :, :n] = wl.gen_tokens(w, "k", s, 1, 0, n)[0]
+        V[s, :, :n] = wl.gen_tokens(w, "v", s, 1, 0, n)[0]
+        Q[s, :, :n] = wl.gen_tokens(w, "q", s, 1, 0, n)[0]
+    cmax = (int(budgets.max()) + 3) // 4 * 4
+    oc = oracle.OracleCache(seqs, w.n_kv_heads, w.group_size, w.head_dim, w.hash_bits, cmax, budgets, w.dtype,
+                            n_sink=w.n_sink, n_recent=w.n_recent, threads=threads)
+    t0 = time.perf_counter()
+    oc.prefill(W, Q, K, V, plens)
+    t_prefill = time.perf_counter() - t0
+    dq = wl.gen_decode_inputs(w, "q", 0, decode_steps)[:, :seqs]
+    dk = wl.gen_decode_inputs(w, "k", 0, decode_steps)[:, :seqs]
+    dv = wl.gen_decode_inputs(w, "v", 0, decode_steps)[:, :seqs]
+    t0 = time.perf_counter()
+    for i in range(decode_steps):
+        oc.step(W, np.ascontiguousarray(dq[i]), np.ascontiguousarray(dk[i]), np.ascontiguousarray(dv[i]))
+    t_decode = time.perf_counter() - t0
+    units = seqs * w.n_kv_heads
+    return {
+        "evictions_per_s": units * decode_steps / t_decode,
+        "prefill_keys_per_s": float(plens.sum()) * w.n_kv_heads / t_prefill,
+        "t_prefill_s": t_prefill, "t_decode_s": t_decode,
+        "sample": f"first {seqs} of {w.n_seq} sequences ({units} units): full prefill, then {decode_steps} decode steps",
+    }
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle timed on the host cores, same metric and config."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    threads = len(os.sched_getaffinity(0))
+    seqs, dsteps = args.ref_seqs, args.ref_decode_steps
+    vals, pf = [], []
+    for i in range(args.warmup + args.steps):
+        r = oracle_sample(w, seqs, dsteps, threads)
+        if i >= args.warmup:
+            vals.append(r["evictions_per_s"])
+            pf.append(r["prefill_keys_per_s"])
+    v = statistics.mean(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * (r["t_prefill_s"] + r["t_decode_s"]), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+        "config": config_dict(w, args.replicas),
+        "prefill_keys_per_s": statistics.mean(pf),
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": r["sample"]},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def config_dict(w, replicas):
+    return {
+        "workload": w.name, "batch": w.batch, "layers_folded": w.layers, "n_kv_heads": w.n_kv_heads,
+        "group_size": w.group_size, "head_dim": w.head_dim, "hash_bits": w.hash_bits, "kv_dtype": w.dtype,
+        "budget": "ragged U[%d,%d]" % (w.budget_lo, w.budget_hi) if w.ragged else w.budget,
+        "prompt_len": "%d x budget" % w.prompt_factor if w.ragged else w.prompt_len,
+        "decode_steps": w.decode_steps, "layer_replicas": replicas, "n_sink": w.n_sink, "n_recent": w.n_recent,
+        "write_scores": True,
+        "l2": "inputs larger than L2: every decode call streams a different layer replica's tables "
+              "(replicas x per-call bytes > 126 MB); prefill reads GBs of prompt",
+    }
+
+
+# ------------------------------------------------------------------------------------------------- ours
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2412_16187_b200 import HashEvictCache, decode_staging_bytes
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    # weak scaling: every rank runs the same shapes on its own seeded shard (independent sequences, no collective)
+    w = w.scaled(seed=w.seed + 1000 * rank)
+    R, T = args.replicas, w.decode_steps
+    B, H, G, d = w.n_seq, w.n_kv_heads, w.group_size, w.head_dim
+    budgets, plens = w.budgets(), w.prompt_lens()
+    Nmax = w.max_prompt_len
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+
+    def up(a):
+        t = torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).cuda(non_blocking=False)
+        return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
+
+    # ---- inputs: generated on the host (seeded), uploaded once; the timed region starts with them in HBM
+    t_gen = time.perf_counter()
+    dK = torch.zeros((B, H, Nmax, d), dtype=tdt, device="cuda")
+    dV = torch.zeros_like(dK)
+    dQ = torch.zeros((B, H * G, Nmax, d), dtype=tdt, device="cuda")
+    for s in range(B):
+        n = int(plens[s])
+        dK[s, :, :n] = up(wl.gen_tokens(w, "k", s, 1, 0, n)[0])
+        dV[s, :, :n] = up(wl.gen_tokens(w, "v", s, 1, 0, n)[0])
+        dQ[s, :, :n] = up(wl.gen_tokens(w, "q", s, 1, 0, n)[0])
+    gq, gk, gv = (up(wl.gen_decode_inputs(w, x, 0, T)) for x in "qkv")
+    dplen = torch.from_numpy(plens).cuda()
+    caches = [HashEvictCache(B, H, G, d, w.hash_bits, budgets, torch.from_numpy(wl.gen_W(w, layer=r)), dtype=tdt,
+                             n_sink=w.n_sink, n_recent=w.n_recent, write_scores=True) for r in range(R)]
+    ws = caches[0].workspace(Nmax)
+    victims = torch.empty((R, B, H), dtype=torch.int32, device="cuda")
+    t_gen = time.perf_counter() - t_gen
+
+    stream = torch.cuda.Stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def prefill_all():
+        for c in caches:
+            c.prefill_compress(dQ, dK, dV, dplen, Nmax, workspace=ws, stream=stream)
+
+    def decode_all():
+        for i in range(T):
+            for r, c in enumerate(caches):
+                c.decode_step(gq[i], gk[i], gv[i], victim_out=victims[r], stream=stream)
+
+    # capture the T x R decode calls once; the library neither allocates nor synchronises, so it is capturable
+    graph = None
+    with torch.cuda.stream(stream):
+        prefill_all()
+        stream.synchronize()
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                decode_all()
+
+    def one_step():
+        e0, e1, e2 = ev(), ev(), ev()
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            prefill_all()
+            e1.record(stream)
+            if graph is not None:
+                graph.replay()
+            else:
+                decode_all()
+            e2.record(stream)
+        return e0, e1, e2
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    t_wall = time.perf_counter()
+    evs = [one_step() for _ in range(args.steps)]
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    clocks = sampler.stop() if rank == 0 else None
+    t_prefill = sum(e0.elapsed_time(e1) for e0, e1, _ in evs) * 1e-3
+    t_decode = sum(e1.elapsed_time(e2) for _, e1, e2 in evs) * 1e-3
+    times = torch.tensor([t_prefill, t_decode, t_prefill + t_decode], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    t_prefill, t_decode, t_total = (float(x) for x in times.cpu())
+
+    K = args.steps
+    units = w.n_units
+    evictions = units * T * R * K * world
+    keys = float(plens.sum()) * H * R * K * world
+    decode_calls = T * R * K
+    value = evictions / t_decode
+    peak, peak_src = measured_peak()
+    dec_bytes = decode_bytes_per_call(w, budgets)
+    pre_bytes = prefill_bytes_per_call(w, budgets, plens)
+    dec_gbs = dec_bytes * decode_calls / t_decode / 1e9
+    pre_gbs = pre_bytes * R * K / t_prefill / 1e9
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+        "ms_per_step": 1e3 * t_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u32", "data": "synthetic", "config": config_dict(w, R),
+        "decode_us_per_call": 1e6 * t_decode / decode_calls,
+        "decode_launch_mode": "cuda graph of he_decode_step calls" if graph is not None else "plain stream launches",
+        "prefill_keys_per_s": keys / t_prefill, "prefill_ms_per_call": 1e3 * t_prefill / (R * K),
+        "roofline": {"kernel": "decode_step_kernel", "bound": "hbm", "achieved": dec_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": dec_gbs / peak, "peak_source": peak_src, "traffic": None,
+                     "algorithmic_bytes_per_launch": dec_bytes},
+        "roofline_prefill": {"call": "he_prefill_compress (hash K, hash Q, replay, gather)", "bound": "hbm",
+                             "achieved": pre_gbs, "peak": peak, "unit": "GB/s", "frac": pre_gbs / peak,
+                             "algorithmic_bytes_per_call": pre_bytes,
+                             "note": "the paper-exact sequential replay is integer-ALU/latency bound, not HBM bound"},
+        "gpu_launches": K * R * (4 + T),
+        "input_setup_s": t_gen,
+    }
+
+    if rank == 0 and not args.skip_e2e:
+        # ---- end to end: host buffers in, victims out, through he_decode_step_host (copies inside the timed region)
+        n_e2e = min(T, args.e2e_steps)
+        hq, hk, hv = (x[:n_e2e].cpu().pin_memory() for x in (gq, gk, gv))
+        hvic = torch.empty((B, H), dtype=torch.int32).pin_memory()
+        staging = torch.empty(decode_staging_bytes(caches[0].cfg), dtype=torch.uint8, device="cuda")
+        for i in range(3):
+            caches[0].decode_step_host(hq[i], hk[i], hv[i], hvic, staging, stream=stream)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            for c in caches:
+                c.decode_step_host(hq[i], hk[i], hv[i], hvic, staging, stream=stream)
+        torch.cuda.synchronize()
+        t_e2e = time.perf_counter() - t0
+        h2d = (hq[0].numel() + hk[0].numel() + hv[0].numel()) * hq.element_size()
+        line["e2e"] = {"value": units * n_e2e * R * world / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                       "d2h_bytes_per_step": hvic.numel() * 4,
+                       "what": f"he_decode_step_host, {n_e2e} decode steps x {R} layer replicas, one call = one step; "
+                               "pinned host q/k/v copied in and victims copied out inside the timed region"}
+
+    if rank == 0:
+        line["clocks"] = clocks
+        if not args.skip_cpu_baseline and world == 1:
+            threads = len(os.sched_getaffinity(0))
+            r = oracle_sample(w, args.ref_seqs, args.ref_decode_steps, threads)
+            line["cpu_baseline"] = {"value": r["evictions_per_s"], "unit": UNIT, "cores": threads, "kind": "oracle",
+                                    "sample": r["sample"], "prefill_keys_per_s": r["prefill_keys_per_s"],
+                                    "seconds": r["t_prefill_s"] + r["t_decode_s"]}
+        line["wall_s_timed_region"] = t_wall
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="throughput_batch", choices=list(wl.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--replicas", type=int, default=None, help="independent layer replicas cycled by the decode loop")
+    ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of a CUDA graph")
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=64)
+    ap.add_argument("--ref-seqs", type=int, default=2, help="sequences in the oracle's bounded sample")
+    ap.add_argument("--ref-decode-steps", type=int, default=64)
+    args = ap.parse_args()
+    w = wl.CONFIGS[args.workload]
+    if args.decode_steps is not None:
+        w = w.scaled(decode_steps=args.decode_steps)
+    if args.replicas is None:
+        args.replicas = DEFAULT_REPLICAS[args.workload]
+    if args.warmup < 3 and args.impl == "ours":
+        print("note: fewer than 3 warm-up steps", file=sys.stderr)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

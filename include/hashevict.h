@@ -1,0 +1,150 @@
+/*
+ * hashevict.h - C ABI of the HashEvict eviction hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library keeps, per (sequence, KV head) "unit", a key/value cache of at most C slots and a
+ * table of b-bit SimHash codes of the cached keys. Each decode step hashes the new query and key,
+ * scores every cached key by Hamming distance to the query code, and overwrites the slot with
+ * the lowest score by the new token (Section 3: Eq. 4-6 and Algorithm 1). The prefill call does
+ * the same for a whole prompt (Section 3, "Prompt Encoding Stage").
+ *
+ * General rules for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller unless a parameter says "host".
+ *     The library allocates no memory; scratch space is passed in by the caller.
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*) and return at once;
+ *     they never synchronise (the *_host variants are the exception and say so). Results are
+ *     valid once the stream has been synchronised.
+ *   - The return value is a status code (HE_OK = 0). No exception crosses this boundary.
+ *     he_last_error() returns a human-readable description of the calling thread's last failure.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails with HE_ERR_CUDA.
+ *
+ * Layouts (B sequences, Hkv KV heads, G query heads per KV head, d = head_dim, b = hash_bits,
+ * Wd = ceil(b/32), Cmax = max_budget = slot stride, unit u = s*Hkv + h):
+ *   k_cache, v_cache  [B, Hkv, Cmax, d]   dtype of the config, rows 16-byte aligned
+ *   codes             [B, Hkv, Cmax, Wd]  uint32; bit i of a code is the sign bit of column i of W,
+ *                                         stored in word i/32 at bit i%32; unused high bits are 0
+ *   scores            [B, Hkv, Cmax]      fp32, -(Hamming distance summed over the group)
+ *   pos               [B, Hkv, Cmax]      int32 token position held by the slot, -1 = empty
+ *   budget            [B]                 int32 C_s <= Cmax, read-only
+ *   fill, next_pos    [B, Hkv]            int32 valid slots / position of the next token, per unit
+ *   W                 [d, b]              fp32 row-major: W = R^T of Eq. 2, read-only while in use
+ */
+#ifndef HASHEVICT_H_
+#define HASHEVICT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  HE_OK = 0,
+  HE_ERR_INVALID_ARG = 1, /* null or misaligned pointer, size out of range */
+  HE_ERR_UNSUPPORTED = 2, /* shape outside what the kernels were built for */
+  HE_ERR_CUDA = 3,        /* a CUDA runtime call or launch failed */
+  HE_ERR_WORKSPACE = 4    /* caller-provided scratch too small */
+};
+
+enum { HE_DTYPE_F32 = 0, HE_DTYPE_BF16 = 1 };
+
+/* flags */
+#define HE_FLAG_WRITE_SCORES 1u /* store the per-slot scores of Eq. 5 on every evicting step */
+
+typedef struct he_config {
+  int32_t batch;      /* B; independent layers may be folded in by the caller */
+  int32_t n_kv_heads; /* Hkv */
+  int32_t group_size; /* G >= 1; the G query heads of a KV head add their Hamming distances */
+  int32_t head_dim;   /* d, a multiple of 8, <= 256 */
+  int32_t hash_bits;  /* b in [1, 64] */
+  int32_t max_budget; /* Cmax: slot stride of the cache arrays, a multiple of 4, <= 2^20 */
+  int32_t n_sink;     /* tokens at positions < n_sink are never evicted (0 = plain Algorithm 1) */
+  int32_t n_recent;   /* the n_recent newest cached tokens are never evicted (0 = plain Algorithm 1) */
+  int32_t dtype;      /* HE_DTYPE_* of q, k, v and of the K/V caches */
+  uint32_t flags;     /* HE_FLAG_* */
+} he_config;
+
+typedef struct he_cache {
+  void* k_cache;
+  void* v_cache;
+  uint32_t* codes;
+  float* scores;
+  int32_t* pos;
+  const int32_t* budget;
+  int32_t* fill;
+  int32_t* next_pos;
+  const float* W;
+} he_cache;
+
+/*
+ * he_hash_keys - SimHash codes of `rows` vectors (keys or queries alike), Eq. 2:
+ *   code bit i of row r = [ sum_c x[r, c] * W[c, i] >= 0 ]   (sgn(0) = 1).
+ * x: [rows, d] with a row stride of `row_stride_elems` elements (>= d, rows 16-byte aligned),
+ * dtype from cfg. codes_out: [rows, Wd] uint32. Only head_dim, hash_bits and dtype of cfg are used.
+ * The projection is accumulated in fp32; a bit may differ from exact arithmetic only where the
+ * exact projection is within 1e-5 * |x| * |W[:, i]| of zero. rows = 0 is a no-op.
+ */
+int he_hash_keys(const he_config* cfg, const void* x, int64_t rows, int64_t row_stride_elems, const float* W,
+                 uint32_t* codes_out, void* stream);
+
+/*
+ * he_decode_step - one application of Algorithm 1, lines 1-5, to every unit ("Decoding Stage").
+ * q: [B, Hkv*G, d], k, v: [B, Hkv, d] (contiguous). For each unit, with t = next_pos:
+ *   cache not full (fill < C_s): the token is appended at slot fill; nothing is scored;
+ *   otherwise D_j = sum_g popcount(codes[j] xor h(q_g)) for every slot (Eq. 5, score_j = -D_j),
+ *   the victim is the lowest-index eligible slot with the largest D_j (Eq. 6); a slot is eligible
+ *   when n_sink <= pos_j < t - n_recent (if no slot is eligible, all are).
+ * Then K, V, code and pos of that slot are overwritten by k, v, h(k), t; next_pos and fill advance.
+ * victim_out [B, Hkv]: slot written. evicted_pos_out [B, Hkv] (nullable): position that was evicted,
+ * -1 when appended. qcodes_out [B, Hkv*G, Wd] (nullable): the query codes that were used.
+ * The scores array is written only with HE_FLAG_WRITE_SCORES.
+ */
+int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
+                   int32_t* victim_out, int32_t* evicted_pos_out, uint32_t* qcodes_out, void* stream);
+
+/*
+ * he_prefill_compress - "Prompt Encoding Stage": the cache is reset, the first C_s prompt tokens fill
+ * slots 0..C_s-1, and every later prompt token t = C_s..N_s-1 goes through Algorithm 1 in order, so
+ * the result equals he_reset followed by N_s calls of he_decode_step.
+ * q: [B, Hkv*G, N, d], k, v: [B, Hkv, N, d] addressed with element strides (batch, head, token);
+ * channels are contiguous and every row is 16-byte aligned. prompt_len: [B] int32 on the device,
+ * each <= max_prompt_len. Queries of tokens that are appended are never read.
+ * workspace: at least he_workspace_bytes(cfg, max_prompt_len) bytes, 256-byte aligned; it receives
+ * the prompt codes: key codes [B*Hkv, Nmax, Wd] followed by query codes [B*Hkv, Nmax, G, Wd]
+ * (query codes of appended tokens are left unwritten). scores hold the last evicting step's values.
+ */
+int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
+                        const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len,
+                        int32_t max_prompt_len, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Scratch bytes he_prefill_compress needs for prompts of up to max_prompt_len tokens (0 on bad input). */
+size_t he_workspace_bytes(const he_config* cfg, int32_t max_prompt_len);
+
+/* he_reset - empty every unit: fill = 0, next_pos = 0, pos = -1, codes = 0, scores = 0. K/V are left as they are. */
+int he_reset(const he_config* cfg, const he_cache* cache, void* stream);
+
+/*
+ * Host-buffer variants: the same calls for callers whose activations live in (preferably pinned)
+ * HOST memory. They copy the inputs to `staging` on `stream`, run the device call, copy the result
+ * back and synchronise `stream` before returning.
+ *   he_decode_step_host:  q/k/v are host pointers laid out as for he_decode_step; victim_host [B, Hkv]
+ *     receives the slots written. staging: >= he_decode_staging_bytes(cfg) device bytes.
+ *   he_prefill_compress_host: q [B, Hkv*G, Nmax, d], k, v [B, Hkv, Nmax, d] contiguous host tensors,
+ *     prompt_len_host [B]; fill_host [B, Hkv] receives the valid-slot counts. staging: >=
+ *     he_prefill_staging_bytes(cfg, max_prompt_len) device bytes (includes the prompt-code workspace).
+ */
+size_t he_decode_staging_bytes(const he_config* cfg);
+int he_decode_step_host(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
+                        const void* v_host, int32_t* victim_host, void* staging, size_t staging_bytes, void* stream);
+size_t he_prefill_staging_bytes(const he_config* cfg, int32_t max_prompt_len);
+int he_prefill_compress_host(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
+                             const void* v_host, const int32_t* prompt_len_host, int32_t max_prompt_len,
+                             int32_t* fill_host, void* staging, size_t staging_bytes, void* stream);
+
+/* Text of the calling thread's most recent error ("" if none). The pointer stays valid until the next failing call. */
+const char* he_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HASHEVICT_H_ */

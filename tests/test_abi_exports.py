@@ -1,0 +1,37 @@
+"""The C ABI library builds, loads without a GPU, and exports every symbol include/hashevict.h declares."""
+import ctypes
+import os
+import re
+
+from paper_2412_16187_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "hashevict.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(he_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_symbols()
+    assert {"he_hash_keys", "he_prefill_compress", "he_decode_step", "he_reset"} <= set(names)
+    L = ctypes.CDLL(build.build_cuda())
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(names) == set(binding.EXPORTS)
+
+
+def test_host_side_validation_needs_no_gpu():
+    L = binding.lib()
+    cfg = binding.he_config(2, 2, 4, 128, 64, 4096, 0, 0, 1, 1)
+    assert L.he_workspace_bytes(ctypes.byref(cfg), 8192) >= 2 * 2 * 8192 * 5 * 2 * 4
+    bad = binding.he_config(2, 2, 4, 128, 65, 4096, 0, 0, 1, 1)
+    assert L.he_workspace_bytes(ctypes.byref(bad), 8192) == 0
+    assert L.he_hash_keys(ctypes.byref(bad), None, 1, 128, None, None, None) == 1
+    assert b"hash_bits" in L.he_last_error()
+    odd = binding.he_config(2, 2, 4, 128, 64, 4098, 0, 0, 1, 1)
+    ca = binding.he_cache()
+    assert L.he_reset(ctypes.byref(odd), ctypes.byref(ca), None) == 1 and b"max_budget" in L.he_last_error()
+    assert L.he_reset(ctypes.byref(cfg), ctypes.byref(ca), None) == 1 and b"null" in L.he_last_error()
