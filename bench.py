@@ -365,6 +365,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--replicas", type=int, default=None, help="independent layer replicas cycled by the decode loop")
     ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--batch", type=int, default=None, help="fewer sequences (profiling captures on a small case)")
+    ap.add_argument("--prompt-factor", type=int, default=None, help="ragged workloads: prompt = factor x budget")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of a CUDA graph")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
@@ -375,6 +377,10 @@ def main():
     w = wl.CONFIGS[args.workload]
     if args.decode_steps is not None:
         w = w.scaled(decode_steps=args.decode_steps)
+    if args.batch is not None:
+        w = w.scaled(batch=args.batch)
+    if args.prompt_factor is not None:
+        w = w.scaled(prompt_factor=args.prompt_factor)
     if args.replicas is None:
         args.replicas = DEFAULT_REPLICAS[args.workload]
     if args.warmup < 3 and args.impl == "ours":
