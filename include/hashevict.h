@@ -74,6 +74,10 @@ typedef struct he_cache {
   int32_t* fill;
   int32_t* next_pos;
   const float* W;
+  const int32_t* budget_host; /* optional HOST copy of budget ([B]), or NULL. When given (and B <= 1024)
+                                 he_decode_step passes the budgets in the kernel parameters, which saves the
+                                 kernel one dependent device read before it can start streaming the code table.
+                                 Must hold the same values as `budget`. */
 } he_cache;
 
 /*

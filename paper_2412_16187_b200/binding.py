@@ -30,7 +30,7 @@ class he_config(ctypes.Structure):
 
 class he_cache(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
-                ("k_cache", "v_cache", "codes", "scores", "pos", "budget", "fill", "next_pos", "W")]
+                ("k_cache", "v_cache", "codes", "scores", "pos", "budget", "fill", "next_pos", "W", "budget_host")]
 
 
 EXPORTS = (
@@ -119,7 +119,7 @@ class HashEvictCache:
     """Device-side cache state (the arrays of he_cache, allocated with torch) plus the calls that act on it."""
 
     def __init__(self, batch, n_kv_heads, group_size, head_dim, hash_bits, budgets, W, dtype=torch.bfloat16,
-                 max_budget=None, n_sink=0, n_recent=0, write_scores=True, device="cuda"):
+                 max_budget=None, n_sink=0, n_recent=0, write_scores=True, device="cuda", host_budget_mirror=True):
         lib()
         dev = torch.device(device)
         budgets = torch.as_tensor(budgets, dtype=torch.int32).reshape(-1)
@@ -141,8 +141,10 @@ class HashEvictCache:
         assert self.W.shape == (head_dim, hash_bits)
         self.cfg = _config(batch, n_kv_heads, group_size, head_dim, hash_bits, cmax, n_sink, n_recent, dtype,
                            HE_FLAG_WRITE_SCORES if write_scores else 0)
+        self._budget_host = (ctypes.c_int32 * batch)(*[int(x) for x in budgets.tolist()])  # host mirror of `budget`
         self.ca = he_cache(*[_ptr(t) for t in (self.k_cache, self.v_cache, self.codes, self.scores, self.pos,
-                                               self.budget, self.fill, self.next_pos, self.W)])
+                                               self.budget, self.fill, self.next_pos, self.W)],
+                           ctypes.cast(self._budget_host, ctypes.c_void_p) if host_budget_mirror else None)
         self._ws = None
 
     # --- the four calls of the boundary -------------------------------------------------------------

@@ -25,9 +25,8 @@ __device__ __forceinline__ uint32_t word_mask(int b, int w) {
   return n >= 32 ? 0xFFFFFFFFu : (n <= 0 ? 0u : ((1u << n) - 1u));
 }
 
-// Copies 16 bytes (8 bf16 or 4 fp32) of a row into fp32 shared memory.
-__device__ __forceinline__ void stage_chunk(float* dst, const void* src_row, int chunk, int dtype) {
-  const uint4 raw = __ldg(reinterpret_cast<const uint4*>(src_row) + chunk);
+// Writes 16 bytes of a row (8 bf16 or 4 fp32, already in registers) to fp32 shared memory.
+__device__ __forceinline__ void store_chunk(float* dst, const uint4 raw, int chunk, int dtype) {
   if (dtype == HE_DTYPE_BF16) {
     float4* o = reinterpret_cast<float4*>(dst + chunk * 8);
     o[0] = make_float4(bf16_bits_to_f32(raw.x & 0xFFFFu), bf16_bits_to_f32(raw.x >> 16), bf16_bits_to_f32(raw.y & 0xFFFFu),
@@ -38,6 +37,11 @@ __device__ __forceinline__ void stage_chunk(float* dst, const void* src_row, int
     *reinterpret_cast<float4*>(dst + chunk * 4) =
         make_float4(__uint_as_float(raw.x), __uint_as_float(raw.y), __uint_as_float(raw.z), __uint_as_float(raw.w));
   }
+}
+
+// Copies 16 bytes (8 bf16 or 4 fp32) of a row into fp32 shared memory.
+__device__ __forceinline__ void stage_chunk(float* dst, const void* src_row, int chunk, int dtype) {
+  store_chunk(dst, __ldg(reinterpret_cast<const uint4*>(src_row) + chunk), chunk, dtype);
 }
 
 // a ? b : c per bit (one LOP3)
@@ -75,6 +79,15 @@ __device__ __forceinline__ Planes4 make_planes4(uint32_t q0, uint32_t q1, uint32
 // Key-dependent half of the group-of-four distance: (D - popc(parity planes)) / 2.
 template <int WORDS>
 __device__ __forceinline__ int half_distance4(const uint32_t (&h)[WORDS], const Planes4 (&p)[WORDS]) {
+  if (WORDS == 2) {
+    // two code words: add the planes of equal weight with carry-save logic first, so three popcounts suffice
+    const uint32_t p1a = bitselect(h[0], p[0].a1, p[0].b1), p1b = bitselect(h[WORDS - 1], p[WORDS - 1].a1, p[WORDS - 1].b1);
+    const uint32_t p2a = bitselect(h[0], p[0].a2, p[0].b2), p2b = bitselect(h[WORDS - 1], p[WORDS - 1].a2, p[WORDS - 1].b2);
+    const uint32_t s1 = p1a ^ p1b, c1 = p1a & p1b;             // weight 1, carry of weight 2
+    const uint32_t s2 = c1 ^ p2a ^ p2b;                          // weight 2
+    const uint32_t c2 = (c1 & p2a) | (c1 & p2b) | (p2a & p2b);  // weight 4
+    return __popc(s1) + 2 * __popc(s2) + 4 * __popc(c2);
+  }
   int d = 0;
 #pragma unroll
   for (int w = 0; w < WORDS; ++w)

@@ -9,9 +9,13 @@
 //      and the arg-max (Eq. 6, lowest index on ties) is a packed-key redux.sync + one block barrier;
 //   4. the victim slot's K, V, code and position are overwritten in place.
 #pragma once
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace he {
+
+constexpr int kMaxBudgetVals = 1024;  // budgets carried in the kernel parameters (4 KB)
 
 struct DecodeArgs {
   he_config cfg;
@@ -22,97 +26,109 @@ struct DecodeArgs {
   int32_t* victim_out;
   int32_t* evicted_pos_out;
   uint32_t* qcodes_out;
+  int n_budget_vals;                       // > 0: budgets are in budget_vals (copied from he_cache.budget_host)
+  int32_t budget_vals[kMaxBudgetVals];
 };
 
 constexpr int kRowBatch = 5;  // rows hashed per pass (G = 4 queries + the key in one pass)
+
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may start while
+// the previous kernel of the stream is still draining. Everything that touches memory another kernel may have
+// written comes after griddep_wait(); only W (read-only while a cache is in use) is read before it.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// -(float)D for a small non-negative integer D without an int->float conversion (a quarter-rate instruction):
+// the bit pattern 0x4B000000 + D is the float 2^23 + D.
+__device__ __forceinline__ float neg_small_int(int D) { return 8388608.0f - __uint_as_float(0x4B000000u + (uint32_t)D); }
 
 template <int WORDS, int GT, int NT>
 __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) decode_step_kernel(const DecodeArgs a) {
   constexpr int SPV = 4 / WORDS;  // slots per 16-byte vector
   constexpr int BP = 32 * WORDS;
+  using Ctx = QueryCtx<WORDS, GT>;
   extern __shared__ __align__(16) uint32_t dsm[];  // the unit's code words
   __shared__ __align__(16) float xs[kRowBatch][kMaxDim];
   __shared__ float part[kMaxDim / kChunk][kRowBatch][BP];
   __shared__ __align__(16) uint32_t codes_s[(kMaxGroup + 1) * WORDS];  // rows 0..G-1: query codes, row G: key code
   __shared__ uint32_t wbest[2][32];
 
+  griddep_launch_dependents();
   const he_config& cfg = a.cfg;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const long long unit = blockIdx.x;
-  const int s = (int)(unit / cfg.n_kv_heads);
+  const int s = blockIdx.y;
+  const int unit = s * cfg.n_kv_heads + blockIdx.x;
   const int d = cfg.head_dim, b = cfg.hash_bits, G = cfg.group_size, es = esize_of(cfg.dtype);
-  const long long Cmax = cfg.max_budget;
-  const int C = a.ca.budget[s];
+  const int Cmax = cfg.max_budget;
+
+  // Hashing work item = (chunk of 32 channels, bit). In the dense shape (b = 32 or 64, whole chunks, one item per
+  // thread, one pass of rows) the thread's 32 values of W are fetched right away: W never changes while a cache
+  // is in use, so this read may overlap the tail of the previous kernel of the stream.
+  const int R = G + 1;
+  const int nch = (d + kChunk - 1) / kChunk;
+  const int nitems = nch * BP;
+  const int cpr = d * es / 16;  // 16-byte chunks per row
+  const bool dense = nitems <= NT && R <= kRowBatch && cpr <= 32;  // one item per thread, one pass, one chunk per lane
+  float wreg[kChunk];
+  if (dense && tid < nitems) {
+    const int c0 = (tid / BP) * kChunk, bi = tid % BP;
+    if (b == BP && d % kChunk == 0) {  // b = 32 or 64 and whole chunks: constant strides, no edge tests
+      const float* wp = a.ca.W + c0 * BP + bi;
+#pragma unroll
+      for (int cc = 0; cc < kChunk; ++cc) wreg[cc] = __ldg(wp + cc * BP);
+    } else {  // columns beyond b and channels beyond d count as zeros
+      const int clen = bi < b ? min(kChunk, d - c0) : 0;
+      const float* wp = a.ca.W + c0 * b + bi;
+#pragma unroll
+      for (int cc = 0; cc < kChunk; ++cc) wreg[cc] = cc < clen ? __ldg(wp + cc * b) : 0.f;
+    }
+  }
+
+  griddep_wait();
+  // The rows to hash are requested before the code table: they head the dependency chain, the table only has to
+  // be there when hashing is done.
+  uint4 xraw = make_uint4(0u, 0u, 0u, 0u);
+  const bool stages = dense && warp < R && lane < cpr;
+  if (stages) {
+    const char* src = warp < G ? static_cast<const char*>(a.q) + ((size_t)unit * G + warp) * d * es
+                               : static_cast<const char*>(a.k) + (size_t)unit * d * es;
+    xraw = __ldg(reinterpret_cast<const uint4*>(src) + lane);
+  }
+  // the new K and V rows, 16 bytes per thread, kept until the victim is known
+  uint4 rowreg = make_uint4(0u, 0u, 0u, 0u);
+  if (tid < 2 * cpr) {
+    const bool is_k = tid < cpr;
+    const char* src = static_cast<const char*>(is_k ? a.k : a.v) + (size_t)unit * d * es;
+    rowreg = __ldg(reinterpret_cast<const uint4*>(src) + (is_k ? tid : tid - cpr));
+  }
+  const int C = min(a.n_budget_vals > 0 ? a.budget_vals[s] : a.ca.budget[s], Cmax);
   const int fill = a.ca.fill[unit];
   const int t = a.ca.next_pos[unit];
-  const bool evict = fill >= C;
 
-  // (1) code words -> shared memory, asynchronously
-  const int nvec = evict ? (C * WORDS + 3) / 4 : 0;
+  // (1) code words -> shared memory, asynchronously. The copy is sized by the budget alone: if the unit turns out
+  // to be still filling (fill < C) the copied words are simply not used.
+  const int nvec = (C * WORDS + 3) / 4;
   {
-    const uint4* cvec = reinterpret_cast<const uint4*>(a.ca.codes + unit * Cmax * WORDS);
+    const uint4* cvec = reinterpret_cast<const uint4*>(a.ca.codes + (size_t)unit * Cmax * WORDS);
     for (int vi = tid; vi < nvec; vi += NT) cp_async16(dsm + 4 * vi, cvec + vi);
     cp_async_commit();
   }
-  // this thread's slice of W for the projection: item = (chunk qd of the channels, bit bi); when there are no more
-  // items than threads (every shape with d <= 128), the 32 values of W are loaded once, before anything is waited on
-  const int nch = (d + kChunk - 1) / kChunk;
-  const int nitems = nch * BP;
-  const bool w_resident = nitems <= NT;
-  float wreg[kChunk];
-  auto load_w = [&](int item) {
-    const int c0 = (item / BP) * kChunk, bi = item % BP;
-#pragma unroll
-    for (int cc = 0; cc < kChunk; ++cc)
-      wreg[cc] = (item < nitems && bi < b && c0 + cc < d) ? __ldg(a.ca.W + (long long)(c0 + cc) * b + bi) : 0.f;
-  };
-  load_w(tid);
-  // the new K and V rows, 16 bytes per thread, kept until the victim is known
-  const int cpr = d * es / 16;
-  uint4 rowreg = make_uint4(0u, 0u, 0u, 0u);
-  if (tid < 2 * cpr) {
-    const char* src = static_cast<const char*>(tid < cpr ? a.k : a.v) + unit * d * es;
-    rowreg = __ldg(reinterpret_cast<const uint4*>(src) + (tid % cpr));
-  }
 
-  // (2) hash the G query rows and the key row (Eq. 2)
-  const int R = G + 1;
-  for (int r0 = 0; r0 < R; r0 += kRowBatch) {
-    for (int idx = tid; idx < kRowBatch * cpr; idx += NT) {
-      const int r = idx / cpr, ch = idx % cpr, row = r0 + r;
+  // (2) hash the G query rows and the key row (Eq. 2): one fmaf chain per row and work item, partial sums combined
+  // through shared memory in chunk order.
+  auto stage_rows = [&](int r0) {  // warp r stages row r0 + r as fp32
+    if (warp < kRowBatch) {
+      const int row = r0 + warp;
       if (row < R) {
-        const char* src = row < G ? static_cast<const char*>(a.q) + (unit * G + row) * d * es
-                                  : static_cast<const char*>(a.k) + unit * d * es;
-        stage_chunk(xs[r], src, ch, cfg.dtype);
+        const char* src = row < G ? static_cast<const char*>(a.q) + ((size_t)unit * G + row) * d * es
+                                  : static_cast<const char*>(a.k) + (size_t)unit * d * es;
+        for (int ch = lane; ch < cpr; ch += 32) stage_chunk(xs[warp], src, ch, cfg.dtype);
       } else {
-        for (int i = 0; i < 16 / es; ++i) xs[r][ch * (16 / es) + i] = 0.f;
+        for (int c = lane; c < d; c += 32) xs[warp][c] = 0.f;
       }
     }
-    __syncthreads();
-    for (int item = tid; item < nitems; item += NT) {
-      if (!w_resident) load_w(item);
-      const int qd = item / BP, bi = item % BP;
-      float acc[kRowBatch];
-#pragma unroll
-      for (int r = 0; r < kRowBatch; ++r) acc[r] = 0.f;
-      const int c0 = qd * kChunk;
-#pragma unroll
-      for (int cc = 0; cc < kChunk; cc += 4) {
-        if (c0 + cc < d) {  // d is a multiple of 8, so a group of four channels is all in or all out
-#pragma unroll
-          for (int r = 0; r < kRowBatch; ++r) {
-            const float4 xv = *reinterpret_cast<const float4*>(&xs[r][c0 + cc]);
-            acc[r] = fmaf(xv.x, wreg[cc], acc[r]);
-            acc[r] = fmaf(xv.y, wreg[cc + 1], acc[r]);
-            acc[r] = fmaf(xv.z, wreg[cc + 2], acc[r]);
-            acc[r] = fmaf(xv.w, wreg[cc + 3], acc[r]);
-          }
-        }
-      }
-#pragma unroll
-      for (int r = 0; r < kRowBatch; ++r) part[qd][r][bi] = acc[r];
-    }
-    __syncthreads();
+  };
+  auto combine = [&](int r0) {  // partial sums -> sign bits, one ballot per (row, code word)
     for (int task = warp; task < kRowBatch * WORDS; task += NT / 32) {
       const int r = task / WORDS, w = task % WORDS;
       float tot = 0.f;
@@ -120,60 +136,145 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) decode_step_kernel(co
       const uint32_t word = __ballot_sync(0xFFFFFFFFu, tot >= 0.f) & word_mask(b, w);
       if (lane == 0 && r0 + r < R) codes_s[(r0 + r) * WORDS + w] = word;
     }
-    cp_async_wait_all();  // (no-op after the first pass) this thread's code copies have landed
+  };
+  if (dense) {
+    const bool active = tid < nitems;
+    const int qd = tid / BP, bi = tid % BP;
+    if (stages) store_chunk(xs[warp], xraw, lane, cfg.dtype);
+    if (warp < kRowBatch)  // zeros for absent rows and for the channels that pad the last chunk
+      for (int c = (warp < R ? d : 0) + lane; c < nch * kChunk; c += 32) xs[warp][c] = 0.f;
     __syncthreads();
+    if (active) {
+      float acc[kRowBatch];
+#pragma unroll
+      for (int r = 0; r < kRowBatch; ++r) acc[r] = 0.f;
+      const float* xb = &xs[0][qd * kChunk];
+#pragma unroll
+      for (int cc = 0; cc < kChunk; cc += 4) {
+#pragma unroll
+        for (int r = 0; r < kRowBatch; ++r) {
+          const float4 xv = *reinterpret_cast<const float4*>(xb + r * kMaxDim + cc);
+          acc[r] = fmaf(xv.x, wreg[cc], acc[r]);
+          acc[r] = fmaf(xv.y, wreg[cc + 1], acc[r]);
+          acc[r] = fmaf(xv.z, wreg[cc + 2], acc[r]);
+          acc[r] = fmaf(xv.w, wreg[cc + 3], acc[r]);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < kRowBatch; ++r) part[qd][r][bi] = acc[r];
+    }
+    __syncthreads();
+    combine(0);
+  } else {
+    for (int r0 = 0; r0 < R; r0 += kRowBatch) {
+      if (r0 > 0) __syncthreads();
+      stage_rows(r0);
+      __syncthreads();
+      for (int item = tid; item < nitems; item += NT) {
+        const int qd = item / BP, bi = item % BP, c0 = qd * kChunk;
+        const int clen = min(kChunk, d - c0);
+        float acc[kRowBatch];
+#pragma unroll
+        for (int r = 0; r < kRowBatch; ++r) acc[r] = 0.f;
+        if (bi < b) {
+          for (int cc = 0; cc < clen; cc += 4) {  // d is a multiple of 8
+            float wv[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) wv[k] = __ldg(a.ca.W + (c0 + cc + k) * b + bi);
+#pragma unroll
+            for (int r = 0; r < kRowBatch; ++r) {
+              const float4 xv = *reinterpret_cast<const float4*>(&xs[r][c0 + cc]);
+              acc[r] = fmaf(xv.x, wv[0], acc[r]);
+              acc[r] = fmaf(xv.y, wv[1], acc[r]);
+              acc[r] = fmaf(xv.z, wv[2], acc[r]);
+              acc[r] = fmaf(xv.w, wv[3], acc[r]);
+            }
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < kRowBatch; ++r) part[qd][r][bi] = acc[r];
+      }
+      __syncthreads();
+      combine(r0);
+    }
   }
-  if (a.qcodes_out != nullptr && tid < G * WORDS) a.qcodes_out[unit * G * WORDS + tid] = codes_s[tid];
+  cp_async_wait_all();  // this thread's code copies have landed
+  __syncthreads();
+  if (a.qcodes_out != nullptr && tid < G * WORDS) a.qcodes_out[(size_t)unit * G * WORDS + tid] = codes_s[tid];
 
   // (3) Eq. 5 / Eq. 6
+  const bool evict = fill >= C;
   int slot = fill;
   if (evict) {
-    QueryCtx<WORDS, GT> ctx;
+    Ctx ctx;
     if (GT == 4) {  // build the bit-plane record in registers
-      uint32_t rec[QueryCtx<WORDS, GT>::kRecWords];
-      QueryCtx<WORDS, GT>::build(rec, codes_s, G);
+      uint32_t rec[Ctx::kRecWords];
+      Ctx::build(rec, codes_s, G);
       ctx.load(rec, G);
     } else {
       ctx.load(codes_s, G);
     }
     const bool prot = cfg.n_sink > 0 || cfg.n_recent > 0;
     const bool write_scores = (cfg.flags & HE_FLAG_WRITE_SCORES) != 0;
-    float* sc = a.ca.scores + unit * Cmax;
-    const int32_t* pp = a.ca.pos + unit * Cmax;
+    float* sc = a.ca.scores + (size_t)unit * Cmax;
+    const int32_t* pp = a.ca.pos + (size_t)unit * Cmax;
+    constexpr uint32_t kKeyBase = (1u << kKeyIdxBits) + kKeyIdxMask;  // key = (rank << 20) + kKeyBase - slot
     uint32_t best_all = 0u, best_el = 0u;
+    // one pass over the unit's vectors; PROT and SCORES are compile-time in each instantiation of the loop body
+    auto scan = [&](auto prot_c, auto scores_c) {
+      constexpr bool PROT = decltype(prot_c)::value, SCORES = decltype(scores_c)::value;
 #pragma unroll 2
-    for (int vi = tid; vi < nvec; vi += NT) {
-      const uint4 cvv = *reinterpret_cast<const uint4*>(dsm + 4 * vi);
-      const uint32_t wds[4] = {cvv.x, cvv.y, cvv.z, cvv.w};
-      const int j0 = vi * SPV;
-      float sv[SPV];
+      for (int vi = tid; vi < nvec; vi += NT) {
+        const uint4 cvv = *reinterpret_cast<const uint4*>(dsm + 4 * vi);
+        const uint32_t wds[4] = {cvv.x, cvv.y, cvv.z, cvv.w};
+        const int j0 = vi * SPV;
+        int rk[SPV];
 #pragma unroll
-      for (int e = 0; e < SPV; ++e) {
-        const int j = j0 + e;
-        uint32_t h[WORDS];
+        for (int e = 0; e < SPV; ++e) {
+          uint32_t h[WORDS];
 #pragma unroll
-        for (int w = 0; w < WORDS; ++w) h[w] = wds[e * WORDS + w];
-        const int rk = ctx.rank(h);
-        sv[e] = -(float)ctx.dist(rk);
-        if (j < C) {
-          const uint32_t key = ((uint32_t)(rk + 1) << kKeyIdxBits) | (kKeyIdxMask - (uint32_t)j);
-          best_all = max(best_all, key);
-          if (prot) {
-            const int p = __ldg(pp + j);
-            if (p >= cfg.n_sink && p < t - cfg.n_recent) best_el = max(best_el, key);
-          }
+          for (int w = 0; w < WORDS; ++w) h[w] = wds[e * WORDS + w];
+          rk[e] = ctx.rank(h);
         }
-      }
-      if (write_scores) {
-        if (j0 + SPV <= C) {
-          if (SPV == 4) *reinterpret_cast<float4*>(sc + j0) = make_float4(sv[0], sv[1], sv[SPV > 2 ? 2 : 0], sv[SPV > 3 ? 3 : 0]);
-          else *reinterpret_cast<float2*>(sc + j0) = make_float2(sv[0], sv[1]);
+        if (j0 + SPV <= C) {  // every vector but possibly a unit's last one
+#pragma unroll
+          for (int e = 0; e < SPV; ++e) {
+            const uint32_t key = ((uint32_t)rk[e] << kKeyIdxBits) + (kKeyBase - (uint32_t)(j0 + e));
+            best_all = max(best_all, key);
+            if (PROT) {
+              const int p = __ldg(pp + j0 + e);
+              if (p >= cfg.n_sink && p < t - cfg.n_recent) best_el = max(best_el, key);
+            }
+          }
+          if (SCORES) {
+            if (SPV == 4)
+              *reinterpret_cast<float4*>(sc + j0) =
+                  make_float4(neg_small_int(ctx.dist(rk[0])), neg_small_int(ctx.dist(rk[1])),
+                              neg_small_int(ctx.dist(rk[SPV > 2 ? 2 : 0])), neg_small_int(ctx.dist(rk[SPV > 3 ? 3 : 0])));
+            else
+              *reinterpret_cast<float2*>(sc + j0) = make_float2(neg_small_int(ctx.dist(rk[0])), neg_small_int(ctx.dist(rk[1])));
+          }
         } else {
 #pragma unroll
           for (int e = 0; e < SPV; ++e)
-            if (j0 + e < C) sc[j0 + e] = sv[e];
+            if (j0 + e < C) {
+              const uint32_t key = ((uint32_t)rk[e] << kKeyIdxBits) + (kKeyBase - (uint32_t)(j0 + e));
+              best_all = max(best_all, key);
+              if (PROT) {
+                const int p = __ldg(pp + j0 + e);
+                if (p >= cfg.n_sink && p < t - cfg.n_recent) best_el = max(best_el, key);
+              }
+              if (SCORES) sc[j0 + e] = neg_small_int(ctx.dist(rk[e]));
+            }
         }
       }
+    };
+    using T = std::true_type;
+    using F = std::false_type;
+    if (prot) {
+      if (write_scores) scan(T{}, T{}); else scan(T{}, F{});
+    } else {
+      if (write_scores) scan(F{}, T{}); else scan(F{}, F{});
     }
     uint32_t fin = block_max_key(best_all, wbest[0], lane, warp, NT / 32);
     if (prot) {
@@ -184,18 +285,20 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) decode_step_kernel(co
   }
 
   // (4) Algorithm 1 lines 2-5: the slot takes the new token's K, V, code and position
+  const size_t slot_idx = (size_t)unit * Cmax + slot;
   if (tid < 2 * cpr) {
-    char* dst = static_cast<char*>(tid < cpr ? a.ca.k_cache : a.ca.v_cache) + (unit * Cmax + slot) * d * es;
-    reinterpret_cast<uint4*>(dst)[tid % cpr] = rowreg;
+    const bool is_k = tid < cpr;
+    char* dst = static_cast<char*>(is_k ? a.ca.k_cache : a.ca.v_cache) + slot_idx * d * es;
+    reinterpret_cast<uint4*>(dst)[is_k ? tid : tid - cpr] = rowreg;
   }
   if (tid == NT - 1) {
     int ev = -1;
-    if (evict && a.evicted_pos_out != nullptr) ev = a.ca.pos[unit * Cmax + slot];
-    a.ca.pos[unit * Cmax + slot] = t;
+    if (evict && a.evicted_pos_out != nullptr) ev = a.ca.pos[slot_idx];
+    a.ca.pos[slot_idx] = t;
 #pragma unroll
-    for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + slot) * WORDS + w] = codes_s[G * WORDS + w];
+    for (int w = 0; w < WORDS; ++w) a.ca.codes[slot_idx * WORDS + w] = codes_s[G * WORDS + w];
     if (!evict) {
-      a.ca.scores[unit * Cmax + slot] = 0.f;
+      a.ca.scores[slot_idx] = 0.f;
       a.ca.fill[unit] = fill + 1;
     }
     a.ca.next_pos[unit] = t + 1;

@@ -12,6 +12,7 @@
 
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -116,27 +117,46 @@ int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments
   return HE_OK;
 }
 
+// Decode launches carry the programmatic-serialization attribute so that consecutive he_decode_step kernels of a
+// stream (or of a captured graph) overlap their launch latency; set HE_DISABLE_PDL=1 to launch them plainly.
+bool pdl_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("HE_DISABLE_PDL");
+    return !(e && e[0] == '1');
+  }();
+  return on;
+}
+
 template <int WORDS, int GT, int NT>
-int launch_decode_one(const DecodeArgs& a, size_t smem, long long units, cudaStream_t stream) {
+int launch_decode_one(const DecodeArgs& a, size_t smem, dim3 grid, cudaStream_t stream) {
   if (int rc = set_smem(decode_step_kernel<WORDS, GT, NT>, smem)) return rc;
-  decode_step_kernel<WORDS, GT, NT><<<(unsigned)units, NT, smem, stream>>>(a);
-  HE_CUDA_CHECK(cudaGetLastError());
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = grid;
+  lc.blockDim = dim3(NT);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = pdl_enabled() ? 1 : 0;
+  HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, decode_step_kernel<WORDS, GT, NT>, a));
   return HE_OK;
 }
 
 template <int WORDS, int GT>
-int launch_decode_nt(const DecodeArgs& a, int nt, size_t smem, long long units, cudaStream_t stream) {
-  if (nt == 256) return launch_decode_one<WORDS, GT, 256>(a, smem, units, stream);
-  if (nt == 512) return launch_decode_one<WORDS, GT, 512>(a, smem, units, stream);
-  return launch_decode_one<WORDS, GT, 1024>(a, smem, units, stream);
+int launch_decode_nt(const DecodeArgs& a, int nt, size_t smem, dim3 grid, cudaStream_t stream) {
+  if (nt == 256) return launch_decode_one<WORDS, GT, 256>(a, smem, grid, stream);
+  if (nt == 512) return launch_decode_one<WORDS, GT, 512>(a, smem, grid, stream);
+  return launch_decode_one<WORDS, GT, 1024>(a, smem, grid, stream);
 }
 
 template <int WORDS>
-int launch_decode_g(const DecodeArgs& a, int nt, size_t smem, long long units, cudaStream_t stream) {
+int launch_decode_g(const DecodeArgs& a, int nt, size_t smem, dim3 grid, cudaStream_t stream) {
   switch (a.cfg.group_size) {
-    case 1: return launch_decode_nt<WORDS, 1>(a, nt, smem, units, stream);
-    case 4: return launch_decode_nt<WORDS, 4>(a, nt, smem, units, stream);
-    default: return launch_decode_nt<WORDS, 0>(a, nt, smem, units, stream);
+    case 1: return launch_decode_nt<WORDS, 1>(a, nt, smem, grid, stream);
+    case 4: return launch_decode_nt<WORDS, 4>(a, nt, smem, grid, stream);
+    default: return launch_decode_nt<WORDS, 0>(a, nt, smem, grid, stream);
   }
 }
 
@@ -227,11 +247,27 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
   int nt = 256;
   if (nvec > 2048) nt = 512;
   if (nvec > 4096) nt = 1024;
-  const long long units = (long long)cfg->batch * cfg->n_kv_heads;
-  if (units > 0x7FFFFFFFLL) return fail(HE_ERR_UNSUPPORTED, "too many units");
-  DecodeArgs a{*cfg, *cache, q, k, v, victim_out, evicted_pos_out, qcodes_out};
+  if (cfg->batch > 65535) return fail(HE_ERR_UNSUPPORTED, "batch %d > 65535 in one decode call", cfg->batch);
+  if ((long long)cfg->batch * cfg->n_kv_heads * cfg->max_budget * Wd > 0x7FFFFFFFLL * 16)
+    return fail(HE_ERR_UNSUPPORTED, "cache too large for one decode call");
+  DecodeArgs a;
+  a.cfg = *cfg;
+  a.ca = *cache;
+  a.q = q;
+  a.k = k;
+  a.v = v;
+  a.victim_out = victim_out;
+  a.evicted_pos_out = evicted_pos_out;
+  a.qcodes_out = qcodes_out;
+  a.n_budget_vals = 0;
+  if (cache->budget_host != nullptr && cfg->batch <= kMaxBudgetVals) {
+    // budgets travel in the kernel parameters, so the code-table copy can start without a dependent device read
+    a.n_budget_vals = cfg->batch;
+    memcpy(a.budget_vals, cache->budget_host, sizeof(int32_t) * (size_t)cfg->batch);
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return Wd == 1 ? launch_decode_g<1>(a, nt, smem, units, st) : launch_decode_g<2>(a, nt, smem, units, st);
+  const dim3 grid((unsigned)cfg->n_kv_heads, (unsigned)cfg->batch);
+  return Wd == 1 ? launch_decode_g<1>(a, nt, smem, grid, st) : launch_decode_g<2>(a, nt, smem, grid, st);
 }
 
 size_t he_workspace_bytes(const he_config* cfg, int32_t max_prompt_len) {
