@@ -145,6 +145,33 @@ int he_prefill_compress_host(const he_config* cfg, const he_cache* cache, const 
                              const void* v_host, const int32_t* prompt_len_host, int32_t max_prompt_len,
                              int32_t* fill_host, void* staging, size_t staging_bytes, void* stream);
 
+/*
+ * he_prefill_compress_noalloc - he_prefill_compress for callers that cannot obtain device memory for the
+ * prompt-code workspace. (The paper has no counterpart: this is a packaging variant, the computation and the
+ * results are those of he_prefill_compress.)
+ *
+ * Who needs it: code that runs where allocating is not possible or not allowed - inside a serving loop whose
+ * memory pool is fully committed to the KV cache, in a plug-in that receives raw pointers but no allocator, or
+ * in a process that must not call cudaMalloc once it has started (allocation synchronises the device and can
+ * fail late). Such callers still pass their inputs and the cache arrays; only the scratch is provided here.
+ *
+ * The scratch is a fixed array of HE_NOALLOC_SCRATCH_BYTES bytes that lives in the library's device image:
+ * every GPU that loads the library holds it until the process exits. The call fails with HE_ERR_WORKSPACE,
+ * and does nothing, when he_workspace_bytes(cfg, max_prompt_len) exceeds that size. It never calls cudaMalloc,
+ * cudaFree or any allocating routine.
+ *
+ * The first call on each device looks up the array's device address (one cudaGetSymbolAddress with that device
+ * current); make that first call outside of any stream capture. All calls share the one array and it keeps
+ * whatever the previous call wrote: nothing in it needs to start at zero, but two calls whose kernels overlap
+ * on the GPU (different streams, no ordering between them) would overwrite each other's prompt codes - order
+ * them on one stream or with events. After the call the prompt codes are in the array only until the next call.
+ * All other arguments, layouts and error codes are those of he_prefill_compress.
+ */
+#define HE_NOALLOC_SCRATCH_BYTES (16u << 20)
+int he_prefill_compress_noalloc(const he_config* cfg, const he_cache* cache, const void* q, const void* k,
+                                const void* v, const int64_t q_strides[3], const int64_t kv_strides[3],
+                                const int32_t* prompt_len, int32_t max_prompt_len, void* stream);
+
 /* Text of the calling thread's most recent error ("" if none). The pointer stays valid until the next failing call. */
 const char* he_last_error(void);
 

@@ -36,7 +36,7 @@ class he_cache(ctypes.Structure):
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
     "he_decode_staging_bytes", "he_decode_step_host", "he_prefill_staging_bytes", "he_prefill_compress_host",
-    "he_last_error",
+    "he_prefill_compress_noalloc", "he_last_error",
 )
 
 _lib = None
@@ -66,10 +66,11 @@ def lib():
     L.he_prefill_staging_bytes.argtypes = [cfgp, i32]
     L.he_prefill_staging_bytes.restype = sz
     L.he_prefill_compress_host.argtypes = [cfgp, cap, vp, vp, vp, vp, i32, vp, vp, sz, vp]
+    L.he_prefill_compress_noalloc.argtypes = [cfgp, cap, vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), vp, i32, vp]
     L.he_last_error.argtypes = []
     L.he_last_error.restype = ctypes.c_char_p
     for name in ("he_hash_keys", "he_decode_step", "he_prefill_compress", "he_reset", "he_decode_step_host",
-                 "he_prefill_compress_host"):
+                 "he_prefill_compress_host", "he_prefill_compress_noalloc"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -175,6 +176,16 @@ class HashEvictCache:
         _check(lib().he_prefill_compress(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q), _ptr(k), _ptr(v),
                                          i64x3(*q.stride()[:3]), i64x3(*k.stride()[:3]), _ptr(prompt_len), nmax,
                                          _ptr(ws), ws.numel(), _stream(stream)))
+
+    def prefill_compress_noalloc(self, q, k, v, prompt_len, max_prompt_len=None, stream=None):
+        """he_prefill_compress_noalloc: same call, prompt codes go to the library's built-in scratch (no workspace,
+        no allocation). Raises HashEvictError when the prompt codes would not fit HE_NOALLOC_SCRATCH_BYTES."""
+        nmax = k.shape[2] if max_prompt_len is None else max_prompt_len
+        assert q.stride(3) == 1 and k.stride(3) == 1 and k.stride() == v.stride()
+        i64x3 = ctypes.c_int64 * 3
+        _check(lib().he_prefill_compress_noalloc(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q), _ptr(k), _ptr(v),
+                                                 i64x3(*q.stride()[:3]), i64x3(*k.stride()[:3]), _ptr(prompt_len), nmax,
+                                                 _stream(stream)))
 
     def prompt_codes(self, max_prompt_len):
         """Views of the prompt codes he_prefill_compress left in the workspace: keys [B, H, Nmax, Wd], queries [B, H, Nmax, G, Wd]."""

@@ -14,6 +14,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 #include "decode_kernels.cuh"
@@ -206,6 +207,10 @@ int launch_replay(const ReplayArgs& a, long long units, cudaStream_t stream) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Scratch of he_prefill_compress_noalloc: part of the device image, so no allocation is ever needed for it.
+// In host code this name is only a handle for the runtime's symbol calls, never a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[HE_NOALLOC_SCRATCH_BYTES];
+
 }  // namespace
 
 extern "C" {
@@ -343,6 +348,35 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
   prefill_gather_kernel<<<dim3((unsigned)gx, (unsigned)units), kGatherThreads, 0, st>>>(ga);
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
+}
+
+int he_prefill_compress_noalloc(const he_config* cfg, const he_cache* cache, const void* q, const void* k,
+                                const void* v, const int64_t q_strides[3], const int64_t kv_strides[3],
+                                const int32_t* prompt_len, int32_t max_prompt_len, void* stream) {
+  if (int rc = check_config(cfg, true)) return rc;
+  if (max_prompt_len < 0) return fail(HE_ERR_INVALID_ARG, "max_prompt_len %d < 0", max_prompt_len);
+  const size_t need = he_workspace_bytes(cfg, max_prompt_len);
+  if (need > HE_NOALLOC_SCRATCH_BYTES)
+    return fail(HE_ERR_WORKSPACE, "prompt codes need %zu bytes, the built-in scratch holds %u; use he_prefill_compress with your own workspace",
+                need, (unsigned)HE_NOALLOC_SCRATCH_BYTES);
+  // device address of the built-in array, looked up once per device with that device current
+  static std::mutex mu;
+  static void* scratch_of_device[64] = {};
+  int dev = 0;
+  HE_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(HE_ERR_UNSUPPORTED, "device index %d", dev);
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (scratch_of_device[dev] == nullptr) {
+      void* p = nullptr;
+      HE_CUDA_CHECK(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+      scratch_of_device[dev] = p;
+    }
+    scratch = scratch_of_device[dev];
+  }
+  return he_prefill_compress(cfg, cache, q, k, v, q_strides, kv_strides, prompt_len, max_prompt_len, scratch,
+                             HE_NOALLOC_SCRATCH_BYTES, stream);
 }
 
 int he_reset(const he_config* cfg, const he_cache* cache, void* stream) {
