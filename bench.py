@@ -286,17 +286,15 @@ def run_ours(args, w):
     clocks = sampler.stop() if rank == 0 else None
     t_prefill = sum(e0.elapsed_time(e1) for e0, e1, _ in evs) * 1e-3
     t_decode = sum(e1.elapsed_time(e2) for _, e1, e2 in evs) * 1e-3
-    times = torch.tensor([t_prefill, t_decode, t_prefill + t_decode], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    t_prefill, t_decode, t_total = (float(x) for x in times.cpu())
+    from paper_2412_16187_b200 import shard
 
     K = args.steps
     units = w.n_units
-    evictions = units * T * R * K * world
-    keys = float(plens.sum()) * H * R * K * world
     decode_calls = T * R * K
-    value = evictions / t_decode
+    # whole job = units of all ranks / max over ranks of the device time (no data-path collective: units are independent)
+    evictions, t_decode, value = shard.job_throughput(float(units * T * R * K), t_decode, device="cuda")
+    keys, t_prefill, prefill_rate = shard.job_throughput(float(plens.sum()) * H * R * K, t_prefill, device="cuda")
+    t_total = t_prefill + t_decode
     peak, peak_src = measured_peak()
     dec_bytes = decode_bytes_per_call(w, budgets)
     pre_bytes = prefill_bytes_per_call(w, budgets, plens)
@@ -309,7 +307,7 @@ def run_ours(args, w):
         "dtype": "u32", "data": "synthetic", "config": config_dict(w, R),
         "decode_us_per_call": 1e6 * t_decode / decode_calls,
         "decode_launch_mode": "cuda graph of he_decode_step calls" if graph is not None else "plain stream launches",
-        "prefill_keys_per_s": keys / t_prefill, "prefill_ms_per_call": 1e3 * t_prefill / (R * K),
+        "prefill_keys_per_s": prefill_rate, "prefill_ms_per_call": 1e3 * t_prefill / (R * K),
         "roofline": {"kernel": "decode_step_kernel", "bound": "hbm", "achieved": dec_gbs, "peak": peak, "unit": "GB/s",
                      "frac": dec_gbs / peak, "peak_source": peak_src, "traffic": None,
                      "algorithmic_bytes_per_launch": dec_bytes},

@@ -144,3 +144,73 @@ def test_host_buffer_variants_match_device_calls():
                            torch.from_numpy(dv).pin_memory(), vb, st)
     assert torch.equal(va.cpu(), vb)
     assert torch.equal(a.gpu.codes, b.gpu.codes) and torch.equal(a.gpu.k_cache, b.gpu.k_cache)
+
+
+def _sampled_full_size_check(w, seqs, decode_steps):
+    """Full-size workload on the device in the launch configuration the benchmark times; the oracle replays only
+    the sampled sequences (all their KV heads) on the device's codes and must reproduce their final state."""
+    import oracle as orc
+    from parity import raw_np, torch_dtype
+    Nmax = w.max_prompt_len
+    W = wl.gen_W(w)
+    plen, budgets = w.prompt_lens(), w.budgets()
+    gpu = HashEvictCache(w.n_seq, w.n_kv_heads, w.group_size, w.head_dim, w.hash_bits, budgets, torch.from_numpy(W),
+                         dtype=torch_dtype(w))
+    tdt = torch_dtype(w)
+    dK = torch.zeros((w.n_seq, w.n_kv_heads, Nmax, w.head_dim), dtype=tdt, device="cuda")
+    dV = torch.zeros_like(dK)
+    dQ = torch.zeros((w.n_seq, w.n_kv_heads * w.group_size, Nmax, w.head_dim), dtype=tdt, device="cuda")
+    for s in range(w.n_seq):
+        n = int(plen[s])
+        dK[s, :, :n] = to_dev(wl.gen_tokens(w, "k", s, 1, 0, n)[0], w)
+        dV[s, :, :n] = to_dev(wl.gen_tokens(w, "v", s, 1, 0, n)[0], w)
+        dQ[s, :, :n] = to_dev(wl.gen_tokens(w, "q", s, 1, 0, n)[0], w)
+    gpu.prefill_compress(dQ, dK, dV, torch.from_numpy(plen).cuda())
+    torch.cuda.synchronize()
+    kc_all, qc_all = gpu.prompt_codes(Nmax)
+    G, Wd = w.group_size, gpu.Wd
+    dq, dk, dv = (wl.gen_decode_inputs(w, x, 0, decode_steps) for x in "qkv")
+    gq, gk, gv = to_dev(dq, w), to_dev(dk, w), to_dev(dv, w)
+    victim = torch.empty((w.n_seq, w.n_kv_heads), dtype=torch.int32, device="cuda")
+    qcodes = torch.empty((w.n_seq, w.n_kv_heads * G, Wd), dtype=torch.int32, device="cuda")
+    oracles = {}
+    for s in seqs:
+        n = int(plen[s])
+        oc = orc.OracleCache(1, w.n_kv_heads, G, w.head_dim, w.hash_bits, gpu.Cmax, budgets[s:s + 1], w.dtype, threads=8)
+        kc = codes_np(kc_all[s:s + 1, :, :n]).copy()
+        qc = codes_np(qc_all[s:s + 1, :, :n]).copy()
+        qc[:, :, :min(n, int(budgets[s]))] = 0
+        Ks, Vs = raw_np(dK[s:s + 1, :, :n]), raw_np(dV[s:s + 1, :, :n])
+        check_hash_stage(Ks[0], W, w.dtype, kc[0])
+        oc.prefill_codes(kc, qc, np.ascontiguousarray(Ks), np.ascontiguousarray(Vs), plen[s:s + 1])
+        oracles[s] = oc
+    for i in range(decode_steps):
+        gpu.decode_step(gq[i], gk[i], gv[i], victim_out=victim, qcodes_out=qcodes)
+        torch.cuda.synchronize()
+        vic = victim.cpu().numpy()
+        gcodes = codes_np(gpu.codes)
+        for s, oc in oracles.items():
+            kc = np.take_along_axis(gcodes[s:s + 1], vic[s:s + 1, :, None, None].astype(np.int64), axis=2)[:, :, 0, :]
+            ovic, _ = oc.step_codes(codes_np(qcodes[s:s + 1]), kc, np.ascontiguousarray(dk[i, s:s + 1]),
+                                    np.ascontiguousarray(dv[i, s:s + 1]))
+            assert np.array_equal(ovic, vic[s:s + 1]), f"victims differ: sequence {s}, decode step {i}"
+    for s, oc in oracles.items():
+        f = int(oc.fill[0, 0])
+        assert np.array_equal(codes_np(gpu.codes[s]), oc.codes[0]) and np.array_equal(gpu.pos[s].cpu().numpy(), oc.pos[0])
+        assert np.array_equal(gpu.scores[s].cpu().numpy(), oc.scores[0])
+        assert np.array_equal(raw_np(gpu.k_cache[s, :, :f]), oc.k_cache[0, :, :f])
+        assert np.array_equal(raw_np(gpu.v_cache[s, :, :f]), oc.v_cache[0, :, :f])
+
+
+def test_full_size_throughput_batch_sampled_sequences():
+    w = wl.CONFIGS["throughput_batch"]
+    b = w.budgets()
+    order = np.argsort(b)
+    _sampled_full_size_check(w, [int(order[0]), int(order[len(order) // 2]), int(order[-1])], decode_steps=4)
+
+
+def test_full_size_long_prefill_sampled_layer():
+    # full per-unit size (32768-token prompt, 9830 slots, 22938 evicting steps), 4 of the 32 folded layers on the
+    # device, one of them replayed by the oracle
+    w = wl.CONFIGS["long_prefill"].scaled(layers=4)
+    _sampled_full_size_check(w, [2], decode_steps=3)
