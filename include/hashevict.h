@@ -172,6 +172,14 @@ int he_prefill_compress_noalloc(const he_config* cfg, const he_cache* cache, con
                                 const void* v, const int64_t q_strides[3], const int64_t kv_strides[3],
                                 const int32_t* prompt_len, int32_t max_prompt_len, void* stream);
 
+/*
+ * he_device_error_count - how many thread blocks of this library's kernels gave up on a bounded device-side
+ * wait since the library was loaded (0 in a healthy process; the kernels never wait without a limit, and a
+ * block that hits one releases what it holds and returns). This call synchronises the device. Returns -1 if the
+ * counter cannot be read. Diagnostic only: the paper has no counterpart.
+ */
+int he_device_error_count(void);
+
 /* Text of the calling thread's most recent error ("" if none). The pointer stays valid until the next failing call. */
 const char* he_last_error(void);
 

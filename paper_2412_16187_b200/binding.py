@@ -36,7 +36,7 @@ class he_cache(ctypes.Structure):
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
     "he_decode_staging_bytes", "he_decode_step_host", "he_prefill_staging_bytes", "he_prefill_compress_host",
-    "he_prefill_compress_noalloc", "he_last_error",
+    "he_prefill_compress_noalloc", "he_device_error_count", "he_last_error",
 )
 
 _lib = None
@@ -67,6 +67,8 @@ def lib():
     L.he_prefill_staging_bytes.restype = sz
     L.he_prefill_compress_host.argtypes = [cfgp, cap, vp, vp, vp, vp, i32, vp, vp, sz, vp]
     L.he_prefill_compress_noalloc.argtypes = [cfgp, cap, vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), vp, i32, vp]
+    L.he_device_error_count.argtypes = []
+    L.he_device_error_count.restype = ctypes.c_int
     L.he_last_error.argtypes = []
     L.he_last_error.restype = ctypes.c_char_p
     for name in ("he_hash_keys", "he_decode_step", "he_prefill_compress", "he_reset", "he_decode_step_host",
@@ -74,6 +76,11 @@ def lib():
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
+
+
+def device_error_count() -> int:
+    """he_device_error_count: thread blocks that gave up on a bounded wait (0 in a healthy process). Synchronises."""
+    return lib().he_device_error_count()
 
 
 def _check(rc: int):

@@ -1,0 +1,321 @@
+// Eq. 2 on many bf16 rows with the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor memory).
+//
+// Why tensor cores here and nowhere else on this path: the projection X[rows, d] * W[d, b] is the one dense
+// contraction, and at b >= 16 its arithmetic intensity (b flop per input byte) puts the CUDA-core kernel on the
+// fp32 FMA pipe instead of on HBM (profiles/: DRAM at ~5 % of peak). Exactness is kept by splitting the fp32 W
+// into three bf16 terms W = W1 + W2 + W3 (each residual is exact in fp32, so the three terms carry all 24
+// significand bits): x is bf16, every product x * W_t is exact, and only the fp32 accumulation rounds. The sign
+// of the result may therefore differ from exact arithmetic only within the same 1e-5 * |x| * |w| band that the
+// fp32 CUDA-core kernel is allowed; the parity tests check every hashed bit against that rule.
+//
+// One persistent CTA per SM, 192 threads, warp-specialised:
+//   warps 0-3  epilogue: tcgen05.ld the 128 x N fp32 accumulator (one row per thread), sign bits -> code words
+//   warp 4     producer: 16-byte cp.async copies of a 128-row tile into 128B-swizzled K-major shared memory
+//   warp 5     one thread issues 3 terms x d/16 tcgen05.mma (M = 128, N = 32|64, K = 16) per tile and commits
+// Four shared-memory stages for X, W's three terms resident in shared memory, two accumulators in tensor memory
+// so the epilogue of tile i overlaps the MMAs of tile i+1. Every wait on an mbarrier is bounded: when a limit is
+// hit the CTA raises a flag, all roles leave their loops, tensor memory is released and the kernel returns.
+#pragma once
+#include "common.cuh"
+#include "hash_kernels.cuh"
+
+namespace he {
+
+constexpr int kTcThreads = 192;
+constexpr int kTcRows = 128;          // rows per tile = MMA M
+constexpr int kTcStages = 4;          // X tiles in flight
+constexpr int kTcLag = 2;             // cp.async groups the producer leaves in flight before publishing a stage
+constexpr uint32_t kTcSpinLimit = 1u << 22;
+
+__device__ int g_tc_error = 0;  // number of CTAs that gave up on a bounded wait (stays 0 in a healthy run)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait. Returns false (and raises the CTA-wide abort flag) when the limit is hit or another role aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kTcSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
+// 32 consecutive fp32 columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_k128(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) /* leading offset (unused with swizzle) */ |
+         ((uint64_t)(1024 >> 4) << 32) /* stride between 8-row groups */ | (1ull << 46) /* descriptor version */ |
+         (2ull << 61) /* SWIZZLE_128B */;
+}
+
+__device__ __forceinline__ uint16_t bf16_rne_bits(float f) {
+  uint32_t u = __float_as_uint(f);
+  if ((u & 0x7F800000u) == 0x7F800000u) return (uint16_t)(u >> 16);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+
+// Which rows a tile covers and where its codes go (same segment rules as hash_rows_kernel).
+struct TcTile {
+  const char* base;
+  long long stride;  // elements between rows
+  long long row0;
+  int nrows;
+  long long out_base, out_stride;
+};
+
+template <int WORDS>
+__device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long long tiles_per_seg, TcTile* o) {
+  const int seg = (int)(t / tiles_per_seg);
+  const long long ti = t % tiles_per_seg;
+  long long r_begin, r_end;
+  if (job.mode == 0) {
+    o->base = static_cast<const char*>(job.x);
+    o->stride = job.row_stride;
+    r_begin = 0;
+    r_end = job.rows;
+    o->out_base = 0;
+    o->out_stride = WORDS;
+  } else {
+    const int s = seg / job.heads, hh = seg % job.heads;
+    const long long N = job.prompt_len[s], C = job.budget[s];
+    o->base = static_cast<const char*>(job.x) + (s * job.s0 + hh * job.s1) * 2;
+    o->stride = job.s2;
+    r_end = N;
+    if (job.mode == 1) {
+      r_begin = 0;
+      o->out_base = ((long long)s * job.Hkv + hh) * job.Nmax * WORDS;
+      o->out_stride = WORDS;
+    } else {
+      r_begin = C < N ? C : N;
+      const long long unit = (long long)s * job.Hkv + hh / job.G;
+      o->out_base = (unit * job.Nmax * job.G + hh % job.G) * WORDS;
+      o->out_stride = (long long)job.G * WORDS;
+    }
+  }
+  o->row0 = r_begin + ti * kTcRows;
+  if (o->row0 >= r_end) return false;
+  o->nrows = (int)((r_end - o->row0) < kTcRows ? (r_end - o->row0) : kTcRows);
+  return true;
+}
+
+// Dynamic shared memory (after rounding the base up to 1024 bytes):
+//   B: 3 terms x KH halves x [N rows x 128 bytes]      A: kTcStages x KH halves x [128 rows x 128 bytes]
+template <int WORDS>
+__global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJob job, long long total_tiles,
+                                                                     long long tiles_per_seg) {
+  constexpr int N = 32 * WORDS;
+  extern __shared__ unsigned char tc_smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[2 * kTcStages + 4];
+  __shared__ uint32_t tmem_base_s;
+  __shared__ volatile int abort_flag;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int d = job.d, b = job.b;
+  const int KH = d / 64;  // 64-channel halves (128 bytes of bf16 each)
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char* Bs = smem;
+  const int b_tile_bytes = N * 128;
+  unsigned char* As = Bs + 3 * KH * b_tile_bytes;  // N * 128 is a multiple of 1024 for N = 32, 64
+  const int a_half_bytes = kTcRows * 128;
+  const int a_stage_bytes = KH * a_half_bytes;
+
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kTcStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kTcStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kTcStages + 2 + a); };
+
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < kTcStages; ++s) {
+      mbar_init(full_bar(s), 32);  // every producer lane arrives once its copies have landed
+      mbar_init(empty_bar(s), 1);  // tcgen05.commit
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);   // tcgen05.commit
+      mbar_init(tempty_bar(a), 4);  // one lane of each epilogue warp
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) {  // tensor memory: two accumulators of N columns each -> 2N columns (a power of two >= 32)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2 * N)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // W -> three bf16 terms, transposed to [bit][channel] (K-major), 128B-swizzled; columns beyond b are zero
+  for (int idx = tid; idx < d * N; idx += kTcThreads) {
+    const int c = idx / N, i = idx % N;
+    const float w = i < b ? __ldg(job.W + (long long)c * b + i) : 0.f;
+    const uint16_t w1 = bf16_rne_bits(w);
+    const float r1 = w - bf16_bits_to_f32(w1);
+    const uint16_t w2 = bf16_rne_bits(r1);
+    const float r2 = r1 - bf16_bits_to_f32(w2);
+    const uint16_t w3 = bf16_rne_bits(r2);
+    const int kh = c / 64, kk = c % 64;
+    const int off = (i / 8) * 1024 + (i % 8) * 128 + (((kk / 8) ^ (i % 8)) * 16) + (kk % 8) * 2;
+    *reinterpret_cast<uint16_t*>(Bs + (0 * KH + kh) * b_tile_bytes + off) = w1;
+    *reinterpret_cast<uint16_t*>(Bs + (1 * KH + kh) * b_tile_bytes + off) = w2;
+    *reinterpret_cast<uint16_t*>(Bs + (2 * KH + kh) * b_tile_bytes + off) = w3;
+  }
+  fence_proxy_async();  // the generic-proxy writes above are read by the tensor core through the async proxy
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ producer
+    int it = 0;                // tiles this CTA has started
+    int published = 0;         // tiles whose stage has been handed to the MMA thread
+    bool ok = true;
+    auto publish = [&]() {
+      fence_proxy_async();
+      mbar_arrive(full_bar(published % kTcStages));
+      ++published;
+    };
+    for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      TcTile tl;
+      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl)) continue;
+      const int s = it % kTcStages;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / kTcStages) & 1) ^ 1, &abort_flag));  // warp-uniform
+      if (!ok) break;
+      unsigned char* a_stage = As + s * a_stage_bytes;
+      const int cpr = d / 8;  // 16-byte chunks per row
+      for (int idx = lane; idx < kTcRows * cpr; idx += 32) {
+        const int r = idx / cpr, c = idx % cpr;
+        const int rs = r < tl.nrows ? r : tl.nrows - 1;  // rows past the end repeat the last row; their codes are not stored
+        const char* src = tl.base + ((tl.row0 + rs) * tl.stride) * 2 + c * 16;
+        unsigned char* dst = a_stage + (c / 8) * a_half_bytes + (r / 8) * 1024 + (r % 8) * 128 + (((c % 8) ^ (r % 8)) * 16);
+        cp_async16(dst, src);
+      }
+      cp_async_commit();
+      ++it;
+      if (it - published > kTcLag) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(kTcLag) : "memory");
+        publish();
+      }
+    }
+    cp_async_wait_all();
+    while (published < it) publish();
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMA issue (one thread)
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) /* fp32 accumulate */ | (1u << 7) /* A bf16 */ | (1u << 10) /* B bf16 */ |
+                             ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kTcRows >> 4) << 24);
+      int it = 0;
+      for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+        TcTile tl;
+        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl)) continue;
+        const int s = it % kTcStages, acc = it & 1;
+        if (!mbar_wait(tempty_bar(acc), ((it >> 1) & 1) ^ 1, &abort_flag)) break;  // epilogue has drained this accumulator
+        if (!mbar_wait(full_bar(s), (it / kTcStages) & 1, &abort_flag)) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(As + s * a_stage_bytes);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * N);
+        bool accumulate = false;
+        for (int term = 2; term >= 0; --term)  // smallest term first
+          for (int kh = 0; kh < KH; ++kh) {
+            const uint32_t b_addr = smem_u32(Bs + (term * KH + kh) * b_tile_bytes);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {  // K = 16 bf16 = 32 bytes per instruction inside the 128-byte swizzle span
+              tc_mma_bf16(d_tmem, umma_desc_k128(a_addr + kh * a_half_bytes + ks * 32), umma_desc_k128(b_addr + ks * 32), idesc,
+                          accumulate);
+              accumulate = true;
+            }
+          }
+        tc_commit(empty_bar(s));    // the stage may be refilled once these MMAs have read it
+        tc_commit(tfull_bar(acc));  // and the accumulator is complete
+        ++it;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 0-3, one row per thread)
+    int it = 0;
+    for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      TcTile tl;
+      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl)) continue;
+      const int acc = it & 1;
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(acc), (it >> 1) & 1, &abort_flag))) break;  // warp-uniform
+      tc_fence_after();
+      uint32_t code[WORDS];
+#pragma unroll
+      for (int w = 0; w < WORDS; ++w) {
+        uint32_t v[32];
+        tc_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * N + w * 32), v);
+        tc_wait_ld();
+        uint32_t word = 0u;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) word |= (__uint_as_float(v[i]) >= 0.f ? 1u : 0u) << i;
+        code[w] = word & word_mask(b, w);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      const int r = warp * 32 + lane;
+      if (r < tl.nrows) {
+        uint32_t* o = job.out + tl.out_base + (tl.row0 + r) * tl.out_stride;
+#pragma unroll
+        for (int w = 0; w < WORDS; ++w) o[w] = code[w];
+      }
+      ++it;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * N) : "memory");
+  }
+  if (tid == 0 && abort_flag) atomicAdd(&g_tc_error, 1);
+}
+
+}  // namespace he

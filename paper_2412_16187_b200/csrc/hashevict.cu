@@ -14,11 +14,14 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <mutex>
+#include <utility>
 
 #include "common.cuh"
 #include "decode_kernels.cuh"
 #include "hash_kernels.cuh"
+#include "hash_tc_kernels.cuh"
 #include "hashevict.h"
 #include "prefill_kernels.cuh"
 
@@ -85,26 +88,68 @@ int check_cache(const he_cache* ca) {
   return HE_OK;
 }
 
-// Dynamic shared memory above the default limit needs a per-function opt-in; it is asked for once per device.
+// Dynamic shared memory above the default limit needs a per-function opt-in; it is asked for once per
+// (device, kernel) and again only if a larger size is needed.
 template <typename K>
 int set_smem(K kernel, size_t bytes) {
-  static size_t granted[64] = {};
+  // static + dynamic shared memory beyond 48 KB needs the opt-in, so ask whenever the sum could exceed it
+  if (bytes <= 24 * 1024) return HE_OK;
+  static std::mutex mu;
+  static std::map<std::pair<int, const void*>, size_t> granted;
   int dev = 0;
   HE_CUDA_CHECK(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return fail(HE_ERR_UNSUPPORTED, "device index %d", dev);
-  // static + dynamic shared memory beyond 48 KB needs the opt-in, so ask whenever the sum could exceed it
-  if (bytes > 24 * 1024 && bytes > granted[dev]) {
+  std::lock_guard<std::mutex> lock(mu);
+  size_t& have = granted[std::make_pair(dev, reinterpret_cast<const void*>(kernel))];
+  if (bytes > have) {
     HE_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
-    granted[dev] = bytes;
+    have = bytes;
   }
   return HE_OK;
 }
 
+bool tc_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("HE_DISABLE_TC");
+    return !(e && e[0] == '1');
+  }();
+  return on;
+}
+
+int sm_count(int* out) {
+  static int cached[64] = {};
+  int dev = 0;
+  HE_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(HE_ERR_UNSUPPORTED, "device index %d", dev);
+  if (cached[dev] == 0) HE_CUDA_CHECK(cudaDeviceGetAttribute(&cached[dev], cudaDevAttrMultiProcessorCount, dev));
+  *out = cached[dev];
+  return HE_OK;
+}
+
+// Eq. 2 on many rows. bf16 rows with d = 64 or 128 go to the tensor-core kernel once there are enough of them to
+// pay for staging the split W per CTA; everything else runs on the CUDA-core kernel.
 int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments, cudaStream_t stream) {
   if (max_rows_per_segment <= 0 || segments <= 0) return HE_OK;
   const int Wd = words_of(job.b);
-  const size_t smem = ((size_t)job.d * 32 * Wd + (size_t)kHashRows * job.d) * sizeof(float);
   const long long tiles = (max_rows_per_segment + kHashRows - 1) / kHashRows;
+  if (tc_enabled() && job.dtype == HE_DTYPE_BF16 && (job.d == 64 || job.d == 128) && tiles * segments >= 64) {
+    static_assert(kTcRows == kHashRows, "both kernels tile rows by 128");
+    const int N = 32 * Wd, KH = job.d / 64;
+    const size_t smem = 1024 + (size_t)3 * KH * N * 128 + (size_t)kTcStages * KH * kTcRows * 128;
+    int sms = 0;
+    if (int rc = sm_count(&sms)) return rc;
+    const long long total = tiles * segments;
+    const unsigned grid = (unsigned)(total < sms ? total : sms);
+    if (Wd == 1) {
+      if (int rc = set_smem(hash_rows_tc_kernel<1>, smem)) return rc;
+      hash_rows_tc_kernel<1><<<grid, kTcThreads, smem, stream>>>(job, total, tiles);
+    } else {
+      if (int rc = set_smem(hash_rows_tc_kernel<2>, smem)) return rc;
+      hash_rows_tc_kernel<2><<<grid, kTcThreads, smem, stream>>>(job, total, tiles);
+    }
+    HE_CUDA_CHECK(cudaGetLastError());
+    return HE_OK;
+  }
+  const size_t smem = ((size_t)job.d * 32 * Wd + (size_t)kHashRows * job.d) * sizeof(float);
   if (tiles > 0x7FFFFFFFLL || segments > 65535) return fail(HE_ERR_UNSUPPORTED, "hash grid too large (%lld x %d)", tiles, segments);
   dim3 grid((unsigned)tiles, (unsigned)segments);
   if (Wd == 1) {
@@ -174,11 +219,26 @@ int launch_replay_smem(const ReplayArgs& a, long long units, cudaStream_t stream
   return HE_OK;
 }
 
+// The register kernel is persistent: as many CTAs as fit the GPU at once, each claiming units from the schedule.
 template <int WORDS, int GT, int SPT, int NT>
 int launch_replay_reg_one(const ReplayArgs& a, long long units, cudaStream_t stream) {
   const size_t smem = (size_t)a.cfg.max_budget * 4;
   if (int rc = set_smem(prefill_replay_reg_kernel<WORDS, GT, SPT, NT>, smem)) return rc;
-  prefill_replay_reg_kernel<WORDS, GT, SPT, NT><<<(unsigned)units, NT, smem, stream>>>(a);
+  static int per_sm[64] = {};
+  int dev = 0, sms = 0;
+  HE_CUDA_CHECK(cudaGetDevice(&dev));
+  if (int rc = sm_count(&sms)) return rc;
+  if (per_sm[dev] == 0) {
+    int n = 0;
+    HE_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, prefill_replay_reg_kernel<WORDS, GT, SPT, NT>, NT, smem));
+    per_sm[dev] = n > 0 ? n : 1;
+  }
+  const int nbins = sms < kMaxBins ? sms : kMaxBins;
+  prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched);
+  HE_CUDA_CHECK(cudaGetLastError());
+  long long grid = (long long)sms * per_sm[dev];
+  if (grid > units) grid = units;
+  prefill_replay_reg_kernel<WORDS, GT, SPT, NT><<<(unsigned)grid, NT, smem, stream>>>(a);
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
 }
@@ -216,6 +276,12 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[HE_NOALLOC_SCRA
 extern "C" {
 
 const char* he_last_error(void) { return g_err; }
+
+int he_device_error_count(void) {
+  int n = 0;
+  if (cudaMemcpyFromSymbol(&n, he::g_tc_error, sizeof(int)) != cudaSuccess) return -1;
+  return n;
+}
 
 int he_hash_keys(const he_config* cfg, const void* x, int64_t rows, int64_t row_stride_elems, const float* W,
                  uint32_t* codes_out, void* stream) {
@@ -281,7 +347,7 @@ size_t he_workspace_bytes(const he_config* cfg, int32_t max_prompt_len) {
   const size_t Wd = words_of(cfg->hash_bits);
   const size_t kbytes = align_up(units * (size_t)max_prompt_len * Wd * 4, 256);
   const size_t qbytes = align_up(units * (size_t)max_prompt_len * cfg->group_size * Wd * 4, 256);
-  return kbytes + qbytes + 256;
+  return kbytes + qbytes + align_up(sched_words((long long)units) * 4, 256) + 256;
 }
 
 int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
@@ -337,7 +403,9 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
   if (int rc = launch_hash(job, max_prompt_len, (int)units * G, st)) return rc;
 
   // phase 2: the sequential replay of Algorithm 1 over the prompt, one CTA per unit
-  ReplayArgs ra{*cfg, *cache, kcodes, qcodes, prompt_len, max_prompt_len, cfg->max_budget};
+  int32_t* sched = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(qcodes) +
+                                              align_up((size_t)units * max_prompt_len * G * Wd * 4, 256));
+  ReplayArgs ra{*cfg, *cache, kcodes, qcodes, prompt_len, max_prompt_len, cfg->max_budget, sched};
   if (int rc = (Wd == 1 ? launch_replay<1>(ra, units, st) : launch_replay<2>(ra, units, st))) return rc;
 
   // phase 3: surviving K / V rows into their slots

@@ -19,6 +19,7 @@ struct ReplayArgs {
   const int32_t* prompt_len;
   long long Nmax;
   int smem_slots;  // slots the shared-memory tables were sized for
+  int32_t* sched;  // unit schedule written by prefill_schedule_kernel (register kernel only)
 };
 
 constexpr int kStepBlock = 32;  // prompt tokens whose query contexts are staged at a time (one per lane of warp 0)
@@ -54,6 +55,153 @@ struct StepStager {
   }
 };
 
+// ------------------------------------------------------------------------------------------------ scheduling
+
+// Replay work is very uneven when budgets are ragged (a unit costs about (N - C) * C slot visits) and a CTA
+// runs one unit at a time, so units are dealt to one bin per SM, largest first, each to the currently lightest
+// bin. A replay CTA drains the bin of the SM it runs on and then helps other bins. The result never depends on
+// which CTA runs which unit; only the time does.
+//
+// sched layout (int32): [0] nbins, [1] units, [2 .. 2+nbins] bin_start (nbins + 1 entries),
+//                       [3+nbins .. 3+2*nbins) cursor, then order[units] (unit ids grouped by bin).
+constexpr int kMaxBins = 256;
+constexpr int kSchedSortMax = 4096;  // more units than this are dealt round-robin (they balance by number)
+constexpr int kSchedThreads = 1024;
+
+__host__ __device__ inline size_t sched_words(long long units) { return 3 + 2 * (size_t)kMaxBins + (size_t)units; }
+
+__global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const he_config cfg, const int32_t* budget,
+                                                                          const int32_t* prompt_len, int nbins,
+                                                                          int32_t* sched) {
+  __shared__ unsigned long long keys[kSchedSortMax];  // (work << 20) | (0xFFFFF - unit), sorted descending
+  __shared__ unsigned long long load[kMaxBins];
+  __shared__ int count[kMaxBins + 1];
+  __shared__ unsigned char bin_of[kSchedSortMax];  // nbins <= 256
+  const int tid = threadIdx.x;
+  const int units = cfg.batch * cfg.n_kv_heads;
+  int32_t* bin_start = sched + 2;
+  int32_t* cursor = sched + 3 + nbins;
+  int32_t* order = sched + 3 + 2 * nbins;
+  if (tid == 0) {
+    sched[0] = nbins;
+    sched[1] = units;
+  }
+  for (int i = tid; i < nbins; i += kSchedThreads) cursor[i] = 0;
+  if (units > kSchedSortMax) {  // plenty of units: round-robin bins
+    for (int b = tid; b <= nbins; b += kSchedThreads) {
+      // bin b holds units b, b + nbins, ...: count = ceil((units - b) / nbins)
+      long long before = 0;
+      for (int k = 0; k < b; ++k) before += (units - k + nbins - 1) / nbins;
+      bin_start[b] = (int)before;
+    }
+    for (int u = tid; u < units; u += kSchedThreads) {
+      const int b = u % nbins;
+      long long before = 0;
+      for (int k = 0; k < b; ++k) before += (units - k + nbins - 1) / nbins;
+      order[before + u / nbins] = u;
+    }
+    return;
+  }
+  int n = 1;
+  while (n < units) n <<= 1;
+  for (int i = tid; i < n; i += kSchedThreads) {
+    unsigned long long key = 0ull;
+    if (i < units) {
+      const int s = i / cfg.n_kv_heads;
+      const long long C = budget[s], N = prompt_len[s];
+      const long long work = N > C ? (N - C) * C + 1 : 1;  // evicting steps x slots scanned
+      key = ((unsigned long long)work << 20) | (unsigned long long)(0xFFFFF - i);
+    }
+    keys[i] = key;
+  }
+  __syncthreads();
+  for (int k = 2; k <= n; k <<= 1)  // bitonic sort, descending
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < n; i += kSchedThreads) {
+        const int l = i ^ j;
+        if (l > i) {
+          const unsigned long long a = keys[i], b = keys[l];
+          const bool desc = (i & k) == 0;
+          if (desc ? a < b : a > b) {
+            keys[i] = b;
+            keys[l] = a;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  for (int i = tid; i < nbins; i += kSchedThreads) {
+    load[i] = 0ull;
+    count[i] = 0;
+  }
+  __syncthreads();
+  if (tid < 32) {  // greedy: next-largest unit to the lightest bin (lowest index on ties)
+    for (int i = 0; i < units; ++i) {
+      unsigned long long best = ~0ull;
+      for (int b = tid; b < nbins; b += 32) {
+        const unsigned long long cand = (load[b] << 8) | (unsigned long long)b;  // loads stay far below 2^56
+        best = cand < best ? cand : best;
+      }
+      for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+        best = other < best ? other : best;
+      }
+      if (tid == 0) {
+        const int b = (int)(best & 0xFF);
+        load[b] += keys[i] >> 20;
+        bin_of[i] = (unsigned char)b;
+        count[b] += 1;
+      }
+      __syncwarp();
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int acc = 0;
+    for (int b = 0; b < nbins; ++b) {
+      bin_start[b] = acc;
+      acc += count[b];
+      count[b] = 0;
+    }
+    bin_start[nbins] = acc;
+    for (int i = 0; i < units; ++i) {  // sorted order, so each bin lists its largest unit first
+      const int b = bin_of[i];
+      order[bin_start[b] + count[b]++] = 0xFFFFF - (int)(keys[i] & 0xFFFFF);
+    }
+  }
+}
+
+// Next unit for this CTA: from the bin of the SM it runs on, else from the first other bin that still has work.
+// Returns -1 when every bin is drained. Called by warp 0; every unit is handed out exactly once.
+__device__ __forceinline__ int claim_unit(int32_t* sched, int lane) {
+  const int nbins = sched[0];
+  const int32_t* bin_start = sched + 2;
+  int32_t* cursor = sched + 3 + nbins;
+  const int32_t* order = sched + 3 + 2 * nbins;
+  unsigned smid;
+  asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+  const int home = (int)(smid % (unsigned)nbins);
+  for (int base = 0; base < nbins; base += 32) {
+    const int b = (home + base + lane) % nbins;
+    const bool in_range = base + lane < nbins;
+    const int cnt = in_range ? bin_start[b + 1] - bin_start[b] : 0;
+    bool avail = in_range && *reinterpret_cast<volatile int32_t*>(cursor + b) < cnt;
+    unsigned m = __ballot_sync(0xFFFFFFFFu, avail);
+    while (m) {
+      const int src = __ffs(m) - 1;
+      int got = -1;
+      if (lane == src) {
+        const int idx = atomicAdd(cursor + b, 1);
+        if (idx < cnt) got = order[bin_start[b] + idx];
+      }
+      got = __shfl_sync(0xFFFFFFFFu, got, src);
+      if (got >= 0) return got;
+      m &= m - 1;  // that bin was drained in the meantime
+    }
+  }
+  return -1;
+}
+
 // ------------------------------------------------------------------------------------------------ registers
 
 template <int WORDS, int GT, int SPT, int NT>
@@ -63,110 +211,153 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) prefill_replay_reg_ke
   extern __shared__ __align__(16) int32_t pos_s[];  // [smem_slots]
   __shared__ uint32_t wbest[2][2][32];
   __shared__ uint32_t stage[2][kStepBlock * Stager::kRec];
+  __shared__ int s_unit;
+  static_assert(SPT <= 32, "the per-thread key packs the register index in 5 bits");
 
   const he_config& cfg = a.cfg;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const long long unit = blockIdx.x;
-  const int s = (int)(unit / cfg.n_kv_heads);
   const int G = cfg.group_size;
   const long long Cmax = cfg.max_budget;
-  const int C = a.ca.budget[s];
-  const int N = a.prompt_len[s];
-  const int fill0 = N < C ? N : C;
-  const uint32_t* kc_u = a.kcodes + unit * a.Nmax * WORDS;
-  const uint32_t* qc_u = a.qcodes + unit * a.Nmax * G * WORDS;
   const bool prot = cfg.n_sink > 0 || cfg.n_recent > 0;
   const bool write_scores = (cfg.flags & HE_FLAG_WRITE_SCORES) != 0;
-  float* sc = a.ca.scores + unit * Cmax;
 
-  // the first C tokens fill the cache in order; slot j lives in register j / NT of thread j % NT
-  uint32_t code[SPT][WORDS];
-#pragma unroll
-  for (int r = 0; r < SPT; ++r) {
-    const int j = r * NT + tid;
-#pragma unroll
-    for (int w = 0; w < WORDS; ++w) code[r][w] = j < fill0 ? __ldg(kc_u + (long long)j * WORDS + w) : 0u;
-    if (j < fill0) pos_s[j] = j;
-  }
+  for (;;) {
+    if (warp == 0) {
+      const int u = claim_unit(a.sched, lane);
+      if (lane == 0) s_unit = u;
+    }
+    __syncthreads();
+    const long long unit = s_unit;
+    if (unit < 0) break;
+    const int s = (int)(unit / cfg.n_kv_heads);
+    const int C = min(a.ca.budget[s], (int)Cmax);
+    const int N = a.prompt_len[s];
+    const int fill0 = N < C ? N : C;
+    const uint32_t* kc_u = a.kcodes + unit * a.Nmax * WORDS;
+    const uint32_t* qc_u = a.qcodes + unit * a.Nmax * G * WORDS;
+    float* sc = a.ca.scores + unit * Cmax;
 
-  Stager st;
-  st.have = false;
-  int buf = 0;
-  if (C < N && warp == 0) {
-    st.prefetch(qc_u, kc_u, C, N, G, lane);
-    st.commit(stage[0], G, lane);
-  }
-  __syncthreads();
+    // the first C tokens fill the cache in order; slot j lives in register j / NT of thread j % NT
+    uint32_t code[SPT][WORDS];
+#pragma unroll
+    for (int r = 0; r < SPT; ++r) {
+      const int j = r * NT + tid;
+#pragma unroll
+      for (int w = 0; w < WORDS; ++w) code[r][w] = j < fill0 ? __ldg(kc_u + (long long)j * WORDS + w) : 0u;
+      if (j < fill0) pos_s[j] = j;
+    }
+    const int nfull = C / NT;             // registers that hold a valid slot in every thread
+    const bool has_tail = tid < C % NT;   // register nfull holds a valid slot in the first C % NT threads
+    const int nregs = (C + NT - 1) / NT;  // registers that hold a valid slot in some thread
+    const uint32_t vmask = (nfull >= 32 ? 0xFFFFFFFFu : ((1u << nfull) - 1u)) | (has_tail ? (1u << nfull) : 0u);  // bit r: slot valid
 
-  int par = 0;
-  for (int t0 = C; t0 < N; t0 += kStepBlock) {
-    const bool more = t0 + kStepBlock < N;
-    if (more && warp == 0) st.prefetch(qc_u, kc_u, t0 + kStepBlock, N, G, lane);
-    const int tend = (N - t0) < kStepBlock ? (N - t0) : kStepBlock;
-    for (int ts = 0; ts < tend; ++ts) {
-      const int t = t0 + ts;
-      const uint32_t* rec = &stage[buf][ts * Stager::kRec];
-      Ctx ctx;
-      ctx.load(rec, G);
-      const bool last = write_scores && (t == N - 1);
-      uint32_t best_all = 0u, best_el = 0u;
+    Stager st;
+    st.have = false;
+    int buf = 0;
+    if (C < N && warp == 0) {
+      st.prefetch(qc_u, kc_u, C, N, G, lane);
+      st.commit(stage[0], G, lane);
+    }
+    __syncthreads();
+
+    int par = 0;
+    for (int t0 = C; t0 < N; t0 += kStepBlock) {
+      const bool more = t0 + kStepBlock < N;
+      if (more && warp == 0) st.prefetch(qc_u, kc_u, t0 + kStepBlock, N, G, lane);
+      const int tend = (N - t0) < kStepBlock ? (N - t0) : kStepBlock;
+      for (int ts = 0; ts < tend; ++ts) {
+        const int t = t0 + ts;
+        const uint32_t* rec = &stage[buf][ts * Stager::kRec];
+        Ctx ctx;
+        ctx.load(rec, G);
+        const bool last = write_scores && (t == N - 1);
+        // thread-local arg-max over its registers: key = rank * 32 + (31 - r), so equal ranks keep the lower slot.
+        // Registers are visited in groups of four. The common step (no protected window, not the scoring step)
+        // is branch-free inside a group; only the group that straddles the budget masks invalid slots.
+        int loc_all = -1, loc_el = -1;
+        if (!prot && !last) {
 #pragma unroll
-      for (int r = 0; r < SPT; ++r) {
-        const int j = r * NT + tid;
-        const int rk = ctx.rank(code[r]);
-        const uint32_t key = j < C ? (((uint32_t)(rk + 1) << kKeyIdxBits) | (kKeyIdxMask - (uint32_t)j)) : 0u;
-        best_all = max(best_all, key);
-        if (prot && j < C) {
-          const int p = pos_s[j];
-          if (p >= cfg.n_sink && p < t - cfg.n_recent) best_el = max(best_el, key);
-        }
-        if (last && j < C) sc[j] = -(float)ctx.dist(rk);
-      }
-      uint32_t fin = block_max_key(best_all, wbest[par][0], lane, warp, NT / 32);
-      if (prot) {
-        best_el = __reduce_max_sync(0xFFFFFFFFu, best_el);
-        if (lane == 0) wbest[par][1][warp] = best_el;
-        __syncthreads();
-        const uint32_t fin_el = __reduce_max_sync(0xFFFFFFFFu, lane < NT / 32 ? wbest[par][1][lane] : 0u);
-        if (fin_el != 0u) fin = fin_el;
-      }
-      const int slot = (int)(kKeyIdxMask - (fin & kKeyIdxMask));
-      if (slot % NT == tid) {  // the slot's own scanning thread rewrites it, so no extra barrier is needed
-        const int rr = slot / NT;
+          for (int g0 = 0; g0 < SPT; g0 += 4) {
+            if (g0 >= nregs) break;  // uniform over the block
+            if (g0 + 4 <= nfull) {
 #pragma unroll
-        for (int r = 0; r < SPT; ++r)
-          if (r == rr) {
+              for (int r = g0; r < g0 + 4 && r < SPT; ++r) loc_all = max(loc_all, ctx.rank(code[r]) * 32 + (31 - r));
+            } else {
 #pragma unroll
-            for (int w = 0; w < WORDS; ++w) code[r][w] = rec[Ctx::kRecWords + w];
+              for (int r = g0; r < g0 + 4 && r < SPT; ++r) {
+                const int key = ctx.rank(code[r]) * 32 + (31 - r);
+                loc_all = max(loc_all, ((vmask >> r) & 1u) ? key : -1);
+              }
+            }
           }
-        pos_s[slot] = t;
+        } else {
+#pragma unroll
+          for (int r = 0; r < SPT; ++r) {
+            if ((vmask >> r) & 1u) {
+              const int rk = ctx.rank(code[r]);
+              const int key = rk * 32 + (31 - r);
+              loc_all = max(loc_all, key);
+              if (prot) {
+                const int p = pos_s[r * NT + tid];
+                if (p >= cfg.n_sink && p < t - cfg.n_recent) loc_el = max(loc_el, key);
+              }
+              if (last) sc[r * NT + tid] = -(float)ctx.dist(rk);
+            }
+          }
+        }
+        // block-wide key = (rank + 1) << 20 | (0xFFFFF - slot); 0 when the thread has no (eligible) slot
+        auto widen = [&](int loc) -> uint32_t {
+          if (loc < 0) return 0u;
+          const int r = 31 - (loc & 31);
+          return ((uint32_t)((loc >> 5) + 1) << kKeyIdxBits) | (kKeyIdxMask - (uint32_t)(r * NT + tid));
+        };
+        uint32_t fin = block_max_key(widen(loc_all), wbest[par][0], lane, warp, NT / 32);
+        if (prot) {
+          uint32_t best_el = __reduce_max_sync(0xFFFFFFFFu, widen(loc_el));
+          if (lane == 0) wbest[par][1][warp] = best_el;
+          __syncthreads();
+          const uint32_t fin_el = __reduce_max_sync(0xFFFFFFFFu, lane < NT / 32 ? wbest[par][1][lane] : 0u);
+          if (fin_el != 0u) fin = fin_el;
+        }
+        const int slot = (int)(kKeyIdxMask - (fin & kKeyIdxMask));
+        if (slot % NT == tid) {  // the slot's own scanning thread rewrites it, so no extra barrier is needed
+          const int rr = slot / NT;
+#pragma unroll
+          for (int r = 0; r < SPT; ++r)
+            if (r == rr) {
+#pragma unroll
+              for (int w = 0; w < WORDS; ++w) code[r][w] = rec[Ctx::kRecWords + w];
+            }
+          pos_s[slot] = t;
+        }
+        par ^= 1;
       }
-      par ^= 1;
+      if (more) {
+        if (warp == 0) st.commit(stage[buf ^ 1], G, lane);
+        __syncthreads();
+        buf ^= 1;
+      }
     }
-    if (more) {
-      if (warp == 0) st.commit(stage[buf ^ 1], G, lane);
-      __syncthreads();
-      buf ^= 1;
-    }
-  }
-  __syncthreads();
+    __syncthreads();
 
-  // final state of the unit; everything beyond `fill` is reset
-  const bool scored = write_scores && N > C;
+    // final state of the unit; everything beyond `fill` is reset
+    const bool scored = write_scores && N > C;
 #pragma unroll
-  for (int r = 0; r < SPT; ++r) {
-    const int j = r * NT + tid;
-    if (j < Cmax) {
-      const bool valid = j < fill0;
+    for (int r = 0; r < SPT; ++r) {
+      const int j = r * NT + tid;
+      if (j < Cmax) {
+        const bool valid = j < fill0;
 #pragma unroll
-      for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = valid ? code[r][w] : 0u;
-      a.ca.pos[unit * Cmax + j] = valid ? pos_s[j] : -1;
-      if (!(valid && scored)) sc[j] = 0.f;
+        for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = valid ? code[r][w] : 0u;
+        a.ca.pos[unit * Cmax + j] = valid ? pos_s[j] : -1;
+        if (!(valid && scored)) sc[j] = 0.f;
+      }
     }
-  }
-  if (tid == 0) {
-    a.ca.fill[unit] = fill0;
-    a.ca.next_pos[unit] = N;
+    if (tid == 0) {
+      a.ca.fill[unit] = fill0;
+      a.ca.next_pos[unit] = N;
+    }
+    __syncthreads();  // pos_s, stage and s_unit are reused by the next unit
   }
 }
 
