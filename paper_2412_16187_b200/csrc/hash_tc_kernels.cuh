@@ -10,12 +10,16 @@
 //
 // One persistent CTA per SM, 192 threads, warp-specialised:
 //   warps 0-3  epilogue: tcgen05.ld the 128 x N fp32 accumulator (one row per thread), sign bits -> code words
-//   warp 4     producer: 16-byte cp.async copies of a 128-row tile into 128B-swizzled K-major shared memory
+//   warp 4     producer: one thread issues a TMA tensor copy per 64-channel half of a 128-row tile (the hardware
+//              applies the 128-byte swizzle and signals the stage's mbarrier with the byte count); when no tensor
+//              map can be built for the caller's strides the warp falls back to 16-byte cp.async copies
 //   warp 5     one thread issues 3 terms x d/16 tcgen05.mma (M = 128, N = 32|64, K = 16) per tile and commits
 // Four shared-memory stages for X, W's three terms resident in shared memory, two accumulators in tensor memory
 // so the epilogue of tile i overlaps the MMAs of tile i+1. Every wait on an mbarrier is bounded: when a limit is
 // hit the CTA raises a flag, all roles leave their loops, tensor memory is released and the kernel returns.
 #pragma once
+#include <cuda.h>  // CUtensorMap (types only; the encoder is fetched through the runtime)
+
 #include "common.cuh"
 #include "hash_kernels.cuh"
 
@@ -56,6 +60,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
   *abort_flag = 1;
   return false;
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// TMA tile copy global -> shared (no multicast), completion counted in bytes on `bar`
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tmap, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -109,6 +124,7 @@ struct TcTile {
   long long row0;
   int nrows;
   long long out_base, out_stride;
+  int c2, c3;  // tensor-map coordinates of the segment (head, sequence)
 };
 
 template <int WORDS>
@@ -123,9 +139,13 @@ __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long lo
     r_end = job.rows;
     o->out_base = 0;
     o->out_stride = WORDS;
+    o->c2 = 0;
+    o->c3 = 0;
   } else {
     const int s = seg / job.heads, hh = seg % job.heads;
     const long long N = job.prompt_len[s], C = job.budget[s];
+    o->c2 = hh;
+    o->c3 = s;
     o->base = static_cast<const char*>(job.x) + (s * job.s0 + hh * job.s1) * 2;
     o->stride = job.s2;
     r_end = N;
@@ -148,9 +168,10 @@ __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long lo
 
 // Dynamic shared memory (after rounding the base up to 1024 bytes):
 //   B: 3 terms x KH halves x [N rows x 128 bytes]      A: kTcStages x KH halves x [128 rows x 128 bytes]
-template <int WORDS>
+template <int WORDS, bool TMA>
 __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJob job, long long total_tiles,
-                                                                     long long tiles_per_seg) {
+                                                                     long long tiles_per_seg,
+                                                                     const __grid_constant__ CUtensorMap tmap) {
   constexpr int N = 32 * WORDS;
   extern __shared__ unsigned char tc_smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * kTcStages + 4];
@@ -176,7 +197,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   if (tid == 0) {
     abort_flag = 0;
     for (int s = 0; s < kTcStages; ++s) {
-      mbar_init(full_bar(s), 32);  // every producer lane arrives once its copies have landed
+      mbar_init(full_bar(s), TMA ? 1 : 32);  // TMA: one arrive + byte count; cp.async: every producer lane arrives
       mbar_init(empty_bar(s), 1);  // tcgen05.commit
     }
     for (int a = 0; a < 2; ++a) {
@@ -211,8 +232,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
 
-  if (warp == 4) {
-    // ------------------------------------------------------------------ producer
+  if (warp == 4 && TMA) {
+    // ------------------------------------------------------------------ producer (TMA, one thread)
+    if (lane == 0) {
+      int it = 0;
+      for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+        TcTile tl;
+        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl)) continue;
+        const int s = it % kTcStages;
+        if (!mbar_wait(empty_bar(s), ((it / kTcStages) & 1) ^ 1, &abort_flag)) break;
+        mbar_arrive_expect_tx(full_bar(s), (uint32_t)a_stage_bytes);
+        // rows past the tensor's extent are filled with zeros by the copy engine; their codes are not stored
+        for (int kh = 0; kh < KH; ++kh)
+          tma_load_4d(smem_u32(As + s * a_stage_bytes + kh * a_half_bytes), &tmap, kh * 64, (int)tl.row0, tl.c2, tl.c3, full_bar(s));
+        ++it;
+      }
+    }
+  } else if (warp == 4) {
+    // ------------------------------------------------------------------ producer (cp.async fallback)
     int it = 0;                // tiles this CTA has started
     int published = 0;         // tiles whose stage has been handed to the MMA thread
     bool ok = true;

@@ -125,6 +125,52 @@ int sm_count(int* out) {
   return HE_OK;
 }
 
+// Tensor map of the rows to hash, as a 4-D bf16 tensor {channel, row or token, head, sequence} with a box of
+// 64 channels x 128 rows and the 128-byte shared-memory swizzle. Returns false when the driver's encoder is not
+// available or rejects the strides (the kernel then stages rows with cp.async instead).
+bool encode_rows_tmap(const HashJob& job, long long max_rows_per_segment, int segments, CUtensorMap* out) {
+  using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn encode = [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      fn = nullptr;
+    return reinterpret_cast<EncodeFn>(fn);
+  }();
+  memset(out, 0, sizeof(*out));
+  if (encode == nullptr || getenv("HE_DISABLE_TMA") != nullptr) return false;
+  cuuint64_t dims[4], strides[3];
+  dims[0] = (cuuint64_t)job.d;
+  if (job.mode == 0) {
+    dims[1] = (cuuint64_t)job.rows;
+    dims[2] = 1;
+    dims[3] = 1;
+    strides[0] = (cuuint64_t)job.row_stride * 2;
+    strides[1] = strides[0] * dims[1];
+    strides[2] = strides[1];
+  } else {
+    dims[1] = (cuuint64_t)max_rows_per_segment;
+    dims[2] = (cuuint64_t)job.heads;
+    dims[3] = (cuuint64_t)(segments / job.heads);
+    strides[0] = (cuuint64_t)job.s2 * 2;
+    strides[1] = (cuuint64_t)job.s1 * 2;
+    strides[2] = (cuuint64_t)job.s0 * 2;
+  }
+  for (int i = 0; i < 3; ++i)
+    if (strides[i] % 16 != 0 || strides[i] >= (1ull << 40)) return false;
+  for (int i = 0; i < 4; ++i)
+    if (dims[i] == 0 || dims[i] > (1ull << 32)) return false;
+  const cuuint32_t box[4] = {64, (cuuint32_t)kTcRows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(job.x), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Eq. 2 on many rows. bf16 rows with d = 64 or 128 go to the tensor-core kernel once there are enough of them to
 // pay for staging the split W per CTA; everything else runs on the CUDA-core kernel.
 int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments, cudaStream_t stream) {
@@ -139,12 +185,24 @@ int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments
     if (int rc = sm_count(&sms)) return rc;
     const long long total = tiles * segments;
     const unsigned grid = (unsigned)(total < sms ? total : sms);
+    alignas(64) CUtensorMap tmap;
+    const bool tma = encode_rows_tmap(job, max_rows_per_segment, segments, &tmap);
     if (Wd == 1) {
-      if (int rc = set_smem(hash_rows_tc_kernel<1>, smem)) return rc;
-      hash_rows_tc_kernel<1><<<grid, kTcThreads, smem, stream>>>(job, total, tiles);
+      if (tma) {
+        if (int rc = set_smem(hash_rows_tc_kernel<1, true>, smem)) return rc;
+        hash_rows_tc_kernel<1, true><<<grid, kTcThreads, smem, stream>>>(job, total, tiles, tmap);
+      } else {
+        if (int rc = set_smem(hash_rows_tc_kernel<1, false>, smem)) return rc;
+        hash_rows_tc_kernel<1, false><<<grid, kTcThreads, smem, stream>>>(job, total, tiles, tmap);
+      }
     } else {
-      if (int rc = set_smem(hash_rows_tc_kernel<2>, smem)) return rc;
-      hash_rows_tc_kernel<2><<<grid, kTcThreads, smem, stream>>>(job, total, tiles);
+      if (tma) {
+        if (int rc = set_smem(hash_rows_tc_kernel<2, true>, smem)) return rc;
+        hash_rows_tc_kernel<2, true><<<grid, kTcThreads, smem, stream>>>(job, total, tiles, tmap);
+      } else {
+        if (int rc = set_smem(hash_rows_tc_kernel<2, false>, smem)) return rc;
+        hash_rows_tc_kernel<2, false><<<grid, kTcThreads, smem, stream>>>(job, total, tiles, tmap);
+      }
     }
     HE_CUDA_CHECK(cudaGetLastError());
     return HE_OK;
