@@ -30,6 +30,7 @@ constexpr int kTcRows = 128;          // rows per tile = MMA M
 constexpr int kTcStages = 4;          // X tiles in flight
 constexpr int kTcLag = 2;             // cp.async groups the producer leaves in flight before publishing a stage
 constexpr uint32_t kTcSpinLimit = 1u << 22;
+constexpr int kTcLenCache = 2048;     // sequences whose prompt length and budget are cached in shared memory
 
 __device__ int g_tc_error = 0;  // number of CTAs that gave up on a bounded wait (stays 0 in a healthy run)
 
@@ -128,7 +129,8 @@ struct TcTile {
 };
 
 template <int WORDS>
-__device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long long tiles_per_seg, TcTile* o) {
+__device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long long tiles_per_seg, TcTile* o,
+                                        const int* s_len, const int* s_bud) {
   const int seg = (int)(t / tiles_per_seg);
   const long long ti = t % tiles_per_seg;
   long long r_begin, r_end;
@@ -143,7 +145,9 @@ __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long lo
     o->c3 = 0;
   } else {
     const int s = seg / job.heads, hh = seg % job.heads;
-    const long long N = job.prompt_len[s], C = job.budget[s];
+    // lengths come from the CTA's shared-memory copy when the batch fits it: skipping an empty tile is then cheap
+    const long long N = s < kTcLenCache ? s_len[s] : job.prompt_len[s];
+    const long long C = s < kTcLenCache ? s_bud[s] : job.budget[s];
     o->c2 = hh;
     o->c3 = s;
     o->base = static_cast<const char*>(job.x) + (s * job.s0 + hh * job.s1) * 2;
@@ -177,6 +181,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   __shared__ __align__(8) unsigned long long bars[2 * kTcStages + 4];
   __shared__ uint32_t tmem_base_s;
   __shared__ volatile int abort_flag;
+  __shared__ int s_len[kTcLenCache], s_bud[kTcLenCache];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = job.d, b = job.b;
@@ -211,6 +216,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (job.mode != 0) {
+    const int nseq = (int)(total_tiles / tiles_per_seg) / job.heads;
+    for (int i = threadIdx.x; i < nseq && i < kTcLenCache; i += kTcThreads) {
+      s_len[i] = job.prompt_len[i];
+      s_bud[i] = job.budget[i];
+    }
+  }
   // W -> three bf16 terms, transposed to [bit][channel] (K-major), 128B-swizzled; columns beyond b are zero
   for (int idx = tid; idx < d * N; idx += kTcThreads) {
     const int c = idx / N, i = idx % N;
@@ -238,7 +250,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
       int it = 0;
       for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
         TcTile tl;
-        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl)) continue;
+        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud)) continue;
         const int s = it % kTcStages;
         if (!mbar_wait(empty_bar(s), ((it / kTcStages) & 1) ^ 1, &abort_flag)) break;
         mbar_arrive_expect_tx(full_bar(s), (uint32_t)a_stage_bytes);
@@ -260,7 +272,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
     };
     for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
       TcTile tl;
-      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl)) continue;
+      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud)) continue;
       const int s = it % kTcStages;
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / kTcStages) & 1) ^ 1, &abort_flag));  // warp-uniform
       if (!ok) break;
@@ -287,27 +299,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) /* fp32 accumulate */ | (1u << 7) /* A bf16 */ | (1u << 10) /* B bf16 */ |
                              ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kTcRows >> 4) << 24);
+      const uint64_t b_desc0 = umma_desc_k128(smem_u32(Bs));
       int it = 0;
       for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
         TcTile tl;
-        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl)) continue;
+        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud)) continue;
         const int s = it % kTcStages, acc = it & 1;
         if (!mbar_wait(tempty_bar(acc), ((it >> 1) & 1) ^ 1, &abort_flag)) break;  // epilogue has drained this accumulator
         if (!mbar_wait(full_bar(s), (it / kTcStages) & 1, &abort_flag)) break;
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(As + s * a_stage_bytes);
+        // Descriptors differ only in their 14-bit start-address field, so each MMA's pair is the tile's base
+        // descriptor plus a small constant: the issuing thread spends a few instructions per MMA, not dozens.
+        const uint64_t a_desc0 = umma_desc_k128(smem_u32(As + s * a_stage_bytes));
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * N);
-        bool accumulate = false;
-        for (int term = 2; term >= 0; --term)  // smallest term first
-          for (int kh = 0; kh < KH; ++kh) {
-            const uint32_t b_addr = smem_u32(Bs + (term * KH + kh) * b_tile_bytes);
+        if (KH == 2) {
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {  // K = 16 bf16 = 32 bytes per instruction inside the 128-byte swizzle span
-              tc_mma_bf16(d_tmem, umma_desc_k128(a_addr + kh * a_half_bytes + ks * 32), umma_desc_k128(b_addr + ks * 32), idesc,
-                          accumulate);
-              accumulate = true;
-            }
-          }
+          for (int term = 2; term >= 0; --term)  // smallest term first
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh)
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks)  // K = 16 bf16 = 32 bytes per instruction inside the 128-byte swizzle span
+                tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)((kh * (kTcRows * 128) + ks * 32) >> 4),
+                            b_desc0 + (uint64_t)(((term * 2 + kh) * (N * 128) + ks * 32) >> 4), idesc,
+                            !(term == 2 && kh == 0 && ks == 0));
+        } else {
+#pragma unroll
+          for (int term = 2; term >= 0; --term)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)((ks * 32) >> 4), b_desc0 + (uint64_t)((term * (N * 128) + ks * 32) >> 4), idesc,
+                          !(term == 2 && ks == 0));
+        }
         tc_commit(empty_bar(s));    // the stage may be refilled once these MMAs have read it
         tc_commit(tfull_bar(acc));  // and the accumulator is complete
         ++it;
@@ -318,7 +340,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
     int it = 0;
     for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
       TcTile tl;
-      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl)) continue;
+      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud)) continue;
       const int acc = it & 1;
       if (!__all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(acc), (it >> 1) & 1, &abort_flag))) break;  // warp-uniform
       tc_fence_after();
