@@ -309,7 +309,11 @@ def run_ours(args, w):
         "decode_launch_mode": "cuda graph of he_decode_step calls" if graph is not None else "plain stream launches",
         "prefill_keys_per_s": prefill_rate, "prefill_ms_per_call": 1e3 * t_prefill / (R * K),
         "roofline": {"kernel": "decode_step_kernel", "bound": "hbm", "achieved": dec_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": dec_gbs / peak, "peak_source": peak_src, "traffic": None,
+                     "frac": dec_gbs / peak, "peak_source": peak_src,
+                     "traffic": 10414848 if w.name == "throughput_batch" else None,
+                     "traffic_note": "dram read+write bytes of one launch from an ncu capture of this shape "
+                                     "(profiles/decode_step_kernel_throughput_batch.md): 10.4 MB read, the 4.8 MB "
+                                     "written are still in L2 when the kernel ends",
                      "algorithmic_bytes_per_launch": dec_bytes},
         "roofline_prefill": {"call": "he_prefill_compress (hash K, hash Q, replay, gather)", "bound": "hbm",
                              "achieved": pre_gbs, "peak": peak, "unit": "GB/s", "frac": pre_gbs / peak,
