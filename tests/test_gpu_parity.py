@@ -214,3 +214,26 @@ def test_full_size_long_prefill_sampled_layer():
     # device, one of them replayed by the oracle
     w = wl.CONFIGS["long_prefill"].scaled(layers=4)
     _sampled_full_size_check(w, [2], decode_steps=3)
+
+
+def test_prefill_with_token_major_strided_inputs():
+    """q/k/v stored [B, N, heads, d] (token-major, as a fused QKV projection writes them) and handed over as strided
+    views: the tensor-core projection's tensor map and the gather must follow the strides."""
+    w = PARITY_CASES["llama3_8b_gqa"].scaled(batch=2, prompt_len=1500, budget=300, decode_steps=0)
+    a, b = Case(w), Case(w)
+    a.prefill()
+    a.compare_state()
+    tm = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)  # same values, token-major storage
+    q, k, v = tm(b.dQ), tm(b.dK), tm(b.dV)
+    assert not k.is_contiguous() and k.stride(2) == w.n_kv_heads * w.head_dim
+    b.gpu.prefill_compress(q, k, v, b.dplen)
+    torch.cuda.synchronize()
+    for name in ("codes", "pos", "fill", "next_pos", "scores", "k_cache", "v_cache"):
+        assert torch.equal(getattr(a.gpu, name), getattr(b.gpu, name)), name
+
+
+def test_no_kernel_gave_up_on_a_bounded_wait():
+    from paper_2412_16187_b200 import device_error_count
+    x = torch.randn(20000, 128, device="cuda").to(torch.bfloat16)
+    hash_keys(x, torch.randn(128, 64, device="cuda"))
+    assert device_error_count() == 0
