@@ -376,6 +376,9 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
   int nt = 256;
   if (nvec > 2048) nt = 512;
   if (nvec > 4096) nt = 1024;
+  if (nvec > 1024LL * kVecsPerThread)
+    return fail(HE_ERR_UNSUPPORTED, "max_budget %d with %d code words exceeds the decode kernel's %d vectors", cfg->max_budget, Wd,
+                1024 * kVecsPerThread);
   if (cfg->batch > 65535) return fail(HE_ERR_UNSUPPORTED, "batch %d > 65535 in one decode call", cfg->batch);
   if ((long long)cfg->batch * cfg->n_kv_heads * cfg->max_budget * Wd > 0x7FFFFFFFLL * 16)
     return fail(HE_ERR_UNSUPPORTED, "cache too large for one decode call");
