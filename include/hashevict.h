@@ -78,6 +78,10 @@ typedef struct he_cache {
                                  he_decode_step passes the budgets in the kernel parameters, which saves the
                                  kernel one dependent device read before it can start streaming the code table.
                                  Must hold the same values as `budget`. */
+  uint32_t* step_scratch;     /* optional device buffer of he_step_scratch_bytes(cfg) bytes, or NULL. When given and
+                                 a step has at least 16384 new rows (B * Hkv * (G + 1)), he_decode_step first hashes
+                                 all of them with the bulk projection kernels into this buffer and the per-unit
+                                 kernel only scans; results are the same as with the single fused kernel. */
 } he_cache;
 
 /*
@@ -120,6 +124,9 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
 int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
                         const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len,
                         int32_t max_prompt_len, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of he_cache.step_scratch: the codes of one decode step's new rows, (G + 1) * Wd words per unit (0 on bad input). */
+size_t he_step_scratch_bytes(const he_config* cfg);
 
 /* Scratch bytes he_prefill_compress needs for prompts of up to max_prompt_len tokens (0 on bad input). */
 size_t he_workspace_bytes(const he_config* cfg, int32_t max_prompt_len);

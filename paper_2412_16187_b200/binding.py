@@ -30,13 +30,13 @@ class he_config(ctypes.Structure):
 
 class he_cache(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
-                ("k_cache", "v_cache", "codes", "scores", "pos", "budget", "fill", "next_pos", "W", "budget_host")]
+                ("k_cache", "v_cache", "codes", "scores", "pos", "budget", "fill", "next_pos", "W", "budget_host", "step_scratch")]
 
 
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
     "he_decode_staging_bytes", "he_decode_step_host", "he_prefill_staging_bytes", "he_prefill_compress_host",
-    "he_prefill_compress_noalloc", "he_device_error_count", "he_last_error",
+    "he_prefill_compress_noalloc", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
 )
 
 _lib = None
@@ -67,6 +67,8 @@ def lib():
     L.he_prefill_staging_bytes.restype = sz
     L.he_prefill_compress_host.argtypes = [cfgp, cap, vp, vp, vp, vp, i32, vp, vp, sz, vp]
     L.he_prefill_compress_noalloc.argtypes = [cfgp, cap, vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), vp, i32, vp]
+    L.he_step_scratch_bytes.argtypes = [cfgp]
+    L.he_step_scratch_bytes.restype = sz
     L.he_device_error_count.argtypes = []
     L.he_device_error_count.restype = ctypes.c_int
     L.he_last_error.argtypes = []
@@ -152,7 +154,10 @@ class HashEvictCache:
         self._budget_host = (ctypes.c_int32 * batch)(*[int(x) for x in budgets.tolist()])  # host mirror of `budget`
         self.ca = he_cache(*[_ptr(t) for t in (self.k_cache, self.v_cache, self.codes, self.scores, self.pos,
                                                self.budget, self.fill, self.next_pos, self.W)],
-                           ctypes.cast(self._budget_host, ctypes.c_void_p) if host_budget_mirror else None)
+                           ctypes.cast(self._budget_host, ctypes.c_void_p) if host_budget_mirror else None, None)
+        # scratch for the bulk-hashed decode step that large batches use (codes of the step's new rows)
+        self.step_scratch = torch.empty(lib().he_step_scratch_bytes(ctypes.byref(self.cfg)), dtype=torch.uint8, device=dev)
+        self.ca.step_scratch = _ptr(self.step_scratch)
         self._ws = None
 
     # --- the four calls of the boundary -------------------------------------------------------------

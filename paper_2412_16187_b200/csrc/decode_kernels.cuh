@@ -26,6 +26,7 @@ struct DecodeArgs {
   int32_t* victim_out;
   int32_t* evicted_pos_out;
   uint32_t* qcodes_out;
+  const uint32_t* new_codes;               // PRE kernels: [B*Hkv*G + B*Hkv, Wd] codes of this step's q rows, then k rows
   int n_budget_vals;                       // > 0: budgets are in budget_vals (copied from he_cache.budget_host)
   int32_t budget_vals[kMaxBudgetVals];
 };
@@ -43,7 +44,11 @@ __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wa
 // the bit pattern 0x4B000000 + D is the float 2^23 + D.
 __device__ __forceinline__ float neg_small_int(int D) { return 8388608.0f - __uint_as_float(0x4B000000u + (uint32_t)D); }
 
-template <int WORDS, int GT, int NT>
+// PRE = true (large batches): the codes of the step's new rows were written to a.new_codes by the bulk projection
+// kernels launched just before this one in the stream, which themselves started only after everything earlier had
+// finished. So the cache state and the step's k / v rows may be read BEFORE griddepcontrol.wait here; only new_codes
+// is read after it.
+template <int WORDS, int GT, int NT, bool PRE>
 __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) decode_step_kernel(const DecodeArgs a) {
   constexpr int SPV = 4 / WORDS;  // slots per 16-byte vector
   constexpr int BP = 32 * WORDS;
@@ -70,7 +75,7 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) decode_step_kernel(co
   const int nch = (d + kChunk - 1) / kChunk;
   const int nitems = nch * BP;
   const int cpr = d * es / 16;  // 16-byte chunks per row
-  const bool dense = nitems <= NT && R <= kRowBatch && cpr <= 32;  // one item per thread, one pass, one chunk per lane
+  const bool dense = !PRE && nitems <= NT && R <= kRowBatch && cpr <= 32;  // one item per thread, one pass, one chunk per lane
   float wreg[kChunk];
   if (dense && tid < nitems) {
     const int c0 = (tid / BP) * kChunk, bi = tid % BP;
@@ -86,7 +91,7 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) decode_step_kernel(co
     }
   }
 
-  griddep_wait();
+  if (!PRE) griddep_wait();
   // The rows to hash are requested before the code table: they head the dependency chain, the table only has to
   // be there when hashing is done.
   uint4 xraw = make_uint4(0u, 0u, 0u, 0u);
@@ -130,6 +135,12 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) decode_step_kernel(co
 
   // (2) hash the G query rows and the key row (Eq. 2): one fmaf chain per row and work item, partial sums combined
   // through shared memory in chunk order.
+  if (PRE) {
+    griddep_wait();
+    const size_t nq = (size_t)gridDim.x * gridDim.y * G;
+    if (tid < G * WORDS) codes_s[tid] = __ldcg(a.new_codes + (size_t)unit * G * WORDS + tid);
+    else if (tid < R * WORDS) codes_s[tid] = __ldcg(a.new_codes + (nq + unit) * WORDS + (tid - G * WORDS));
+  }
   auto stage_rows = [&](int r0) {  // warp r stages row r0 + r as fp32
     if (warp < kRowBatch) {
       const int row = r0 + warp;
@@ -151,7 +162,9 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) decode_step_kernel(co
       if (lane == 0 && r0 + r < R) codes_s[(r0 + r) * WORDS + w] = word;
     }
   };
-  if (dense) {
+  if (PRE) {
+    // nothing to hash in this kernel
+  } else if (dense) {
     const bool active = tid < nitems;
     const int qd = tid / BP, bi = tid % BP;
     if (stages) store_chunk(xs[warp], xraw, lane, cfg.dtype);

@@ -107,6 +107,8 @@ int set_smem(K kernel, size_t bytes) {
   return HE_OK;
 }
 
+constexpr long long kSplitDecodeRows = 16384;  // new rows per step from which he_decode_step hashes them in bulk first
+
 bool tc_enabled() {
   static const bool on = [] {
     const char* e = getenv("HE_DISABLE_TC");
@@ -231,9 +233,9 @@ bool pdl_enabled() {
   return on;
 }
 
-template <int WORDS, int GT, int NT>
+template <int WORDS, int GT, int NT, bool PRE>
 int launch_decode_one(const DecodeArgs& a, size_t smem, dim3 grid, cudaStream_t stream) {
-  if (int rc = set_smem(decode_step_kernel<WORDS, GT, NT>, smem)) return rc;
+  if (int rc = set_smem(decode_step_kernel<WORDS, GT, NT, PRE>, smem)) return rc;
   cudaLaunchConfig_t lc{};
   lc.gridDim = grid;
   lc.blockDim = dim3(NT);
@@ -244,15 +246,20 @@ int launch_decode_one(const DecodeArgs& a, size_t smem, dim3 grid, cudaStream_t 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
   lc.numAttrs = pdl_enabled() ? 1 : 0;
-  HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, decode_step_kernel<WORDS, GT, NT>, a));
+  HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, decode_step_kernel<WORDS, GT, NT, PRE>, a));
   return HE_OK;
 }
 
 template <int WORDS, int GT>
 int launch_decode_nt(const DecodeArgs& a, int nt, size_t smem, dim3 grid, cudaStream_t stream) {
-  if (nt == 256) return launch_decode_one<WORDS, GT, 256>(a, smem, grid, stream);
-  if (nt == 512) return launch_decode_one<WORDS, GT, 512>(a, smem, grid, stream);
-  return launch_decode_one<WORDS, GT, 1024>(a, smem, grid, stream);
+  if (a.new_codes != nullptr) {
+    if (nt == 256) return launch_decode_one<WORDS, GT, 256, true>(a, smem, grid, stream);
+    if (nt == 512) return launch_decode_one<WORDS, GT, 512, true>(a, smem, grid, stream);
+    return launch_decode_one<WORDS, GT, 1024, true>(a, smem, grid, stream);
+  }
+  if (nt == 256) return launch_decode_one<WORDS, GT, 256, false>(a, smem, grid, stream);
+  if (nt == 512) return launch_decode_one<WORDS, GT, 512, false>(a, smem, grid, stream);
+  return launch_decode_one<WORDS, GT, 1024, false>(a, smem, grid, stream);
 }
 
 template <int WORDS>
@@ -392,12 +399,35 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
   a.evicted_pos_out = evicted_pos_out;
   a.qcodes_out = qcodes_out;
   a.n_budget_vals = 0;
+  a.new_codes = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // Large batches: hash the step's new rows with the bulk projection kernels (tensor cores for bf16) into the
+  // caller's scratch, so the per-unit kernel only scans. Small batches keep the single fused kernel.
+  const long long units_ll = (long long)cfg->batch * cfg->n_kv_heads;
+  if (cache->step_scratch != nullptr && units_ll * (cfg->group_size + 1) >= kSplitDecodeRows &&
+      getenv("HE_DISABLE_SPLIT_DECODE") == nullptr) {
+    HashJob job{};
+    job.W = cache->W;
+    job.mode = 0;
+    job.dtype = cfg->dtype;
+    job.d = cfg->head_dim;
+    job.b = cfg->hash_bits;
+    job.row_stride = cfg->head_dim;
+    job.x = q;
+    job.rows = units_ll * cfg->group_size;
+    job.out = cache->step_scratch;
+    if (int rc = launch_hash(job, job.rows, 1, st)) return rc;
+    job.x = k;
+    job.out = cache->step_scratch + job.rows * Wd;
+    job.rows = units_ll;
+    if (int rc = launch_hash(job, job.rows, 1, st)) return rc;
+    a.new_codes = cache->step_scratch;
+  }
   if (cache->budget_host != nullptr && cfg->batch <= kMaxBudgetVals) {
     // budgets travel in the kernel parameters, so the code-table copy can start without a dependent device read
     a.n_budget_vals = cfg->batch;
     memcpy(a.budget_vals, cache->budget_host, sizeof(int32_t) * (size_t)cfg->batch);
   }
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid((unsigned)cfg->n_kv_heads, (unsigned)cfg->batch);
   return Wd == 1 ? launch_decode_g<1>(a, nt, smem, grid, st) : launch_decode_g<2>(a, nt, smem, grid, st);
 }
@@ -516,6 +546,11 @@ int he_reset(const he_config* cfg, const he_cache* cache, void* stream) {
   reset_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(*cfg, *cache);
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
+}
+
+size_t he_step_scratch_bytes(const he_config* cfg) {
+  if (check_config(cfg, true) != HE_OK) return 0;
+  return (size_t)cfg->batch * cfg->n_kv_heads * (cfg->group_size + 1) * words_of(cfg->hash_bits) * 4;
 }
 
 size_t he_decode_staging_bytes(const he_config* cfg) {

@@ -74,7 +74,6 @@ __global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const h
                                                                           const int32_t* prompt_len, int nbins,
                                                                           int32_t* sched) {
   __shared__ unsigned long long keys[kSchedSortMax];  // (work << 20) | (0xFFFFF - unit), sorted descending
-  __shared__ unsigned long long load[kMaxBins];
   __shared__ int count[kMaxBins + 1];
   __shared__ unsigned char bin_of[kSchedSortMax];  // nbins <= 256
   const int tid = threadIdx.x;
@@ -130,29 +129,37 @@ __global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const h
       }
       __syncthreads();
     }
-  for (int i = tid; i < nbins; i += kSchedThreads) {
-    load[i] = 0ull;
-    count[i] = 0;
-  }
+  for (int i = tid; i < nbins; i += kSchedThreads) count[i] = 0;
   __syncthreads();
   if (tid < 32) {  // greedy: next-largest unit to the lightest bin (lowest index on ties)
+    // Bin loads live in registers (lane l owns bins l, l + 32, ...), scaled to 23 bits so that (load << 8 | bin) fits
+    // one word and the lightest bin is a single redux.sync. The scaling only affects balance, never correctness.
+    constexpr int kOwn = kMaxBins / 32;
+    unsigned long long total = 0ull;
+    for (int i = tid; i < units; i += 32) total += keys[i] >> 20;
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
+    int shift = 0;
+    while ((total >> shift) >= (1ull << 23)) ++shift;
+    uint32_t own[kOwn];
+#pragma unroll
+    for (int k = 0; k < kOwn; ++k) own[k] = 0u;
     for (int i = 0; i < units; ++i) {
-      unsigned long long best = ~0ull;
-      for (int b = tid; b < nbins; b += 32) {
-        const unsigned long long cand = (load[b] << 8) | (unsigned long long)b;  // loads stay far below 2^56
-        best = cand < best ? cand : best;
+      uint32_t best = 0xFFFFFFFFu;
+#pragma unroll
+      for (int k = 0; k < kOwn; ++k) {
+        const int bb = tid + 32 * k;
+        if (bb < nbins) best = min(best, (own[k] << 8) | (uint32_t)bb);
       }
-      for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, best, o);
-        best = other < best ? other : best;
-      }
+      best = __reduce_min_sync(0xFFFFFFFFu, best);
+      const int bb = (int)(best & 0xFFu);
+      const uint32_t wk = (uint32_t)((keys[i] >> 20) >> shift);
+#pragma unroll
+      for (int k = 0; k < kOwn; ++k)
+        if (bb == tid + 32 * k) own[k] += wk;
       if (tid == 0) {
-        const int b = (int)(best & 0xFF);
-        load[b] += keys[i] >> 20;
-        bin_of[i] = (unsigned char)b;
-        count[b] += 1;
+        bin_of[i] = (unsigned char)bb;
+        count[bb] += 1;
       }
-      __syncwarp();
     }
   }
   __syncthreads();

@@ -237,3 +237,13 @@ def test_no_kernel_gave_up_on_a_bounded_wait():
     x = torch.randn(20000, 128, device="cuda").to(torch.bfloat16)
     hash_keys(x, torch.randn(128, 64, device="cuda"))
     assert device_error_count() == 0
+
+
+def test_large_batch_decode_hashes_new_rows_in_bulk():
+    """4096 units x (G + 1) = 20480 new rows per step: he_decode_step hashes them with the bulk projection kernels
+    into the step scratch and the per-unit kernel only scans. Results must not depend on that choice."""
+    w = wl.CONFIGS["throughput_batch"].scaled(batch=512, budget_lo=40, budget_hi=64, prompt_factor=1, decode_steps=5)
+    case = Case(w)
+    case.prefill()
+    case.compare_state()
+    case.decode(5)
