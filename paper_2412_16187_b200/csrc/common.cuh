@@ -44,8 +44,15 @@ __device__ __forceinline__ void stage_chunk(float* dst, const void* src_row, int
   store_chunk(dst, __ldg(reinterpret_cast<const uint4*>(src_row) + chunk), chunk, dtype);
 }
 
-// a ? b : c per bit (one LOP3)
-__device__ __forceinline__ uint32_t bitselect(uint32_t a, uint32_t b, uint32_t c) { return (a & b) | (~a & c); }
+// One LOP3 with an explicit truth table (a = 0xF0, b = 0xCC, c = 0xAA).
+template <int LUT>
+__device__ __forceinline__ uint32_t lop3(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, %4;" : "=r"(d) : "r"(a), "r"(b), "r"(c), "n"(LUT));
+  return d;
+}
+// a ? b : c per bit
+__device__ __forceinline__ uint32_t bitselect(uint32_t a, uint32_t b, uint32_t c) { return lop3<0xCA>(a, b, c); }
 
 // ---------------------------------------------------------------------------------------------------------------
 // Eq. 5 for a group of four query heads without four XOR+popcount passes.
@@ -83,9 +90,9 @@ __device__ __forceinline__ int half_distance4(const uint32_t (&h)[WORDS], const 
     // two code words: add the planes of equal weight with carry-save logic first, so three popcounts suffice
     const uint32_t p1a = bitselect(h[0], p[0].a1, p[0].b1), p1b = bitselect(h[WORDS - 1], p[WORDS - 1].a1, p[WORDS - 1].b1);
     const uint32_t p2a = bitselect(h[0], p[0].a2, p[0].b2), p2b = bitselect(h[WORDS - 1], p[WORDS - 1].a2, p[WORDS - 1].b2);
-    const uint32_t s1 = p1a ^ p1b, c1 = p1a & p1b;             // weight 1, carry of weight 2
-    const uint32_t s2 = c1 ^ p2a ^ p2b;                          // weight 2
-    const uint32_t c2 = (c1 & p2a) | (c1 & p2b) | (p2a & p2b);  // weight 4
+    const uint32_t s1 = p1a ^ p1b, c1 = p1a & p1b;  // weight 1, carry of weight 2
+    const uint32_t s2 = lop3<0x96>(c1, p2a, p2b);     // weight 2: three-way xor
+    const uint32_t c2 = lop3<0xE8>(c1, p2a, p2b);     // weight 4: majority
     return __popc(s1) + 2 * __popc(s2) + 4 * __popc(c2);
   }
   int d = 0;
