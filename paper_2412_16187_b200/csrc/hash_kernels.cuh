@@ -22,6 +22,7 @@ struct HashJob {
   long long Nmax;
   const int32_t* prompt_len;
   const int32_t* budget;
+  const void* w_image;  // optional: the tensor-core kernel's shared-memory image of W's three bf16 terms (build_w_image_kernel)
 };
 
 template <int WORDS>

@@ -118,6 +118,30 @@ __device__ __forceinline__ uint16_t bf16_rne_bits(float f) {
   return (uint16_t)(u >> 16);
 }
 
+// One element of W -> its three bf16 terms at their places in the image (term-major, then 64-channel half, then the
+// [N rows x 128 bytes] K-major tile with the 128-byte swizzle).
+__device__ __forceinline__ void w_image_element(const float* W, int d, int b, int N, int idx, unsigned char* image) {
+  const int c = idx / N, i = idx % N, KH = d / 64, tile_bytes = N * 128;
+  const float w = i < b ? __ldg(W + (long long)c * b + i) : 0.f;
+  const uint16_t w1 = bf16_rne_bits(w);
+  const float r1 = w - bf16_bits_to_f32(w1);
+  const uint16_t w2 = bf16_rne_bits(r1);
+  const float r2 = r1 - bf16_bits_to_f32(w2);
+  const uint16_t w3 = bf16_rne_bits(r2);
+  const int kh = c / 64, kk = c % 64;
+  const int off = (i / 8) * 1024 + (i % 8) * 128 + (((kk / 8) ^ (i % 8)) * 16) + (kk % 8) * 2;
+  *reinterpret_cast<uint16_t*>(image + (0 * KH + kh) * tile_bytes + off) = w1;
+  *reinterpret_cast<uint16_t*>(image + (1 * KH + kh) * tile_bytes + off) = w2;
+  *reinterpret_cast<uint16_t*>(image + (2 * KH + kh) * tile_bytes + off) = w3;
+}
+
+// The image in global memory, built once per call when the caller has scratch for it (kWImageBytes at most).
+constexpr size_t kWImageBytes = 3 * 2 * 64 * 128;  // three terms, d = 128, N = 64
+__global__ void build_w_image_kernel(const float* W, int d, int b, int N, unsigned char* image) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < d * N) w_image_element(W, d, b, N, idx, image);
+}
+
 // Which rows a tile covers and where its codes go (same segment rules as hash_rows_kernel).
 struct TcTile {
   const char* base;
@@ -223,20 +247,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
       s_bud[i] = job.budget[i];
     }
   }
-  // W -> three bf16 terms, transposed to [bit][channel] (K-major), 128B-swizzled; columns beyond b are zero
-  for (int idx = tid; idx < d * N; idx += kTcThreads) {
-    const int c = idx / N, i = idx % N;
-    const float w = i < b ? __ldg(job.W + (long long)c * b + i) : 0.f;
-    const uint16_t w1 = bf16_rne_bits(w);
-    const float r1 = w - bf16_bits_to_f32(w1);
-    const uint16_t w2 = bf16_rne_bits(r1);
-    const float r2 = r1 - bf16_bits_to_f32(w2);
-    const uint16_t w3 = bf16_rne_bits(r2);
-    const int kh = c / 64, kk = c % 64;
-    const int off = (i / 8) * 1024 + (i % 8) * 128 + (((kk / 8) ^ (i % 8)) * 16) + (kk % 8) * 2;
-    *reinterpret_cast<uint16_t*>(Bs + (0 * KH + kh) * b_tile_bytes + off) = w1;
-    *reinterpret_cast<uint16_t*>(Bs + (1 * KH + kh) * b_tile_bytes + off) = w2;
-    *reinterpret_cast<uint16_t*>(Bs + (2 * KH + kh) * b_tile_bytes + off) = w3;
+  // W -> three bf16 terms, transposed to [bit][channel] (K-major), 128B-swizzled; columns beyond b are zero.
+  // Either copied from an image that a one-block-per-slice kernel prepared once for this call, or built here.
+  if (job.w_image != nullptr) {
+    const uint4* src = static_cast<const uint4*>(job.w_image);
+    uint4* dst = reinterpret_cast<uint4*>(Bs);
+    for (int i = tid; i < 3 * KH * b_tile_bytes / 16; i += kTcThreads) dst[i] = __ldg(src + i);
+  } else {
+    for (int idx = tid; idx < d * N; idx += kTcThreads) w_image_element(job.W, d, b, N, idx, Bs);
   }
   fence_proxy_async();  // the generic-proxy writes above are read by the tensor core through the async proxy
   tc_fence_before();

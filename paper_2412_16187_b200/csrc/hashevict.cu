@@ -175,7 +175,7 @@ bool encode_rows_tmap(const HashJob& job, long long max_rows_per_segment, int se
 
 // Eq. 2 on many rows. bf16 rows with d = 64 or 128 go to the tensor-core kernel once there are enough of them to
 // pay for staging the split W per CTA; everything else runs on the CUDA-core kernel.
-int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments, cudaStream_t stream) {
+int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments, cudaStream_t stream, bool* image_built = nullptr) {
   if (max_rows_per_segment <= 0 || segments <= 0) return HE_OK;
   const int Wd = words_of(job.b);
   const long long tiles = (max_rows_per_segment + kHashRows - 1) / kHashRows;
@@ -189,6 +189,12 @@ int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments
     const unsigned grid = (unsigned)(total < sms ? total : sms);
     alignas(64) CUtensorMap tmap;
     const bool tma = encode_rows_tmap(job, max_rows_per_segment, segments, &tmap);
+    if (job.w_image != nullptr && (image_built == nullptr || !*image_built)) {  // scratch of kWImageBytes: filled once per call
+      build_w_image_kernel<<<(job.d * N + 255) / 256, 256, 0, stream>>>(job.W, job.d, job.b, N,
+                                                                       static_cast<unsigned char*>(const_cast<void*>(job.w_image)));
+      HE_CUDA_CHECK(cudaGetLastError());
+      if (image_built != nullptr) *image_built = true;
+    }
     if (Wd == 1) {
       if (tma) {
         if (int rc = set_smem(hash_rows_tc_kernel<1, true>, smem)) return rc;
@@ -413,14 +419,17 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
     job.d = cfg->head_dim;
     job.b = cfg->hash_bits;
     job.row_stride = cfg->head_dim;
+    job.w_image = reinterpret_cast<char*>(cache->step_scratch) +
+                  align_up((size_t)units_ll * (cfg->group_size + 1) * Wd * 4, 256);
     job.x = q;
     job.rows = units_ll * cfg->group_size;
     job.out = cache->step_scratch;
-    if (int rc = launch_hash(job, job.rows, 1, st)) return rc;
+    bool image_built = false;
+    if (int rc = launch_hash(job, job.rows, 1, st, &image_built)) return rc;
     job.x = k;
     job.out = cache->step_scratch + job.rows * Wd;
     job.rows = units_ll;
-    if (int rc = launch_hash(job, job.rows, 1, st)) return rc;
+    if (int rc = launch_hash(job, job.rows, 1, st, &image_built)) return rc;
     a.new_codes = cache->step_scratch;
   }
   if (cache->budget_host != nullptr && cfg->batch <= kMaxBudgetVals) {
@@ -438,7 +447,7 @@ size_t he_workspace_bytes(const he_config* cfg, int32_t max_prompt_len) {
   const size_t Wd = words_of(cfg->hash_bits);
   const size_t kbytes = align_up(units * (size_t)max_prompt_len * Wd * 4, 256);
   const size_t qbytes = align_up(units * (size_t)max_prompt_len * cfg->group_size * Wd * 4, 256);
-  return kbytes + qbytes + align_up(sched_words((long long)units) * 4, 256) + 256;
+  return kbytes + qbytes + align_up(sched_words((long long)units) * 4, 256) + align_up(kWImageBytes, 256) + 256;
 }
 
 int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
@@ -465,8 +474,11 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
   uint32_t* qcodes = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) +
                                                  align_up((size_t)units * max_prompt_len * Wd * 4, 256));
 
+  bool image_built = false;
   // phase 1: Eq. 2 on every prompt key and on the queries of the tokens that will evict
   HashJob job{};
+  job.w_image = static_cast<char*>(workspace) + align_up((size_t)units * max_prompt_len * Wd * 4, 256) +
+                align_up((size_t)units * max_prompt_len * G * Wd * 4, 256) + align_up(sched_words(units) * 4, 256);
   job.W = cache->W;
   job.dtype = cfg->dtype;
   job.d = cfg->head_dim;
@@ -483,7 +495,7 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
   job.s0 = kv_strides[0];
   job.s1 = kv_strides[1];
   job.s2 = kv_strides[2];
-  if (int rc = launch_hash(job, max_prompt_len, (int)units, st)) return rc;
+  if (int rc = launch_hash(job, max_prompt_len, (int)units, st, &image_built)) return rc;
   job.x = q;
   job.out = qcodes;
   job.mode = 2;
@@ -491,7 +503,7 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
   job.s0 = q_strides[0];
   job.s1 = q_strides[1];
   job.s2 = q_strides[2];
-  if (int rc = launch_hash(job, max_prompt_len, (int)units * G, st)) return rc;
+  if (int rc = launch_hash(job, max_prompt_len, (int)units * G, st, &image_built)) return rc;
 
   // phase 2: the sequential replay of Algorithm 1 over the prompt, one CTA per unit
   int32_t* sched = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(qcodes) +
@@ -550,7 +562,8 @@ int he_reset(const he_config* cfg, const he_cache* cache, void* stream) {
 
 size_t he_step_scratch_bytes(const he_config* cfg) {
   if (check_config(cfg, true) != HE_OK) return 0;
-  return (size_t)cfg->batch * cfg->n_kv_heads * (cfg->group_size + 1) * words_of(cfg->hash_bits) * 4;
+  return align_up((size_t)cfg->batch * cfg->n_kv_heads * (cfg->group_size + 1) * words_of(cfg->hash_bits) * 4, 256) +
+         align_up(kWImageBytes, 256);
 }
 
 size_t he_decode_staging_bytes(const he_config* cfg) {
