@@ -223,4 +223,10 @@ __device__ __forceinline__ void cp_async_wait_pending(int pending) {
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;\n" ::: "memory"); }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may start while
+// the previous kernel of the stream is still draining. Everything that touches memory another kernel may have
+// written comes after griddep_wait(); only W (read-only while a cache is in use) is read before it.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 }  // namespace he

@@ -34,12 +34,6 @@ struct DecodeArgs {
 constexpr int kVecsPerThread = 8;  // 16-byte code vectors per thread (the host picks the block size accordingly)
 constexpr int kRowBatch = 5;  // rows hashed per pass (G = 4 queries + the key in one pass)
 
-// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may start while
-// the previous kernel of the stream is still draining. Everything that touches memory another kernel may have
-// written comes after griddep_wait(); only W (read-only while a cache is in use) is read before it.
-__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 // -(float)D for a small non-negative integer D without an int->float conversion (a quarter-rate instruction):
 // the bit pattern 0x4B000000 + D is the float 2^23 + D.
 __device__ __forceinline__ float neg_small_int(int D) { return 8388608.0f - __uint_as_float(0x4B000000u + (uint32_t)D); }
@@ -49,14 +43,15 @@ __device__ __forceinline__ float neg_small_int(int D) { return 8388608.0f - __ui
 // finished. So the cache state and the step's k / v rows may be read BEFORE griddepcontrol.wait here; only new_codes
 // is read after it.
 template <int WORDS, int GT, int NT, bool PRE>
-__global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) decode_step_kernel(const DecodeArgs a) {
+__global__ void __launch_bounds__(NT, (NT <= 256 ? (PRE ? 6 : 4) : 1)) decode_step_kernel(const DecodeArgs a) {
   constexpr int SPV = 4 / WORDS;  // slots per 16-byte vector
   constexpr int BP = 32 * WORDS;
   constexpr bool kGroupedCopy = WORDS == 2;
   using Ctx = QueryCtx<WORDS, GT>;
   extern __shared__ __align__(16) uint32_t dsm[];  // the unit's code words
-  __shared__ __align__(16) float xs[kRowBatch][kMaxDim];
-  __shared__ float part[kMaxDim / kChunk][kRowBatch][BP];
+  // staging of the rows to hash and of the partial sums: not needed when the codes come pre-hashed
+  __shared__ __align__(16) float xs[PRE ? 1 : kRowBatch][PRE ? 4 : kMaxDim];
+  __shared__ float part[PRE ? 1 : kMaxDim / kChunk][PRE ? 1 : kRowBatch][PRE ? 1 : BP];
   __shared__ __align__(16) uint32_t codes_s[(kMaxGroup + 1) * WORDS];  // rows 0..G-1: query codes, row G: key code
   __shared__ uint32_t wbest[2][32];
 

@@ -207,6 +207,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   __shared__ volatile int abort_flag;
   __shared__ int s_len[kTcLenCache], s_bud[kTcLenCache];
 
+  // Programmatic dependent launch (used by the large-batch decode step): a kernel launched behind this one may
+  // start right away; this kernel in turn finishes only after the kernel before it has (see the end).
+  griddep_launch_dependents();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = job.d, b = job.b;
   const int KH = d / 64;  // 64-channel halves (128 bytes of bf16 each)
@@ -393,6 +396,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * N) : "memory");
   }
   if (tid == 0 && abort_flag) atomicAdd(&g_tc_error, 1);
+  griddep_wait();  // no-op unless this kernel was launched programmatically behind another one
 }
 
 }  // namespace he

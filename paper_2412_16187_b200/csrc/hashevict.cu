@@ -109,6 +109,16 @@ int set_smem(K kernel, size_t bytes) {
 
 constexpr long long kSplitDecodeRows = 16384;  // new rows per step from which he_decode_step hashes them in bulk first
 
+// Decode launches carry the programmatic-serialization attribute so that consecutive he_decode_step kernels of a
+// stream (or of a captured graph) overlap their launch latency; set HE_DISABLE_PDL=1 to launch them plainly.
+bool pdl_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("HE_DISABLE_PDL");
+    return !(e && e[0] == '1');
+  }();
+  return on;
+}
+
 bool tc_enabled() {
   static const bool on = [] {
     const char* e = getenv("HE_DISABLE_TC");
@@ -175,7 +185,8 @@ bool encode_rows_tmap(const HashJob& job, long long max_rows_per_segment, int se
 
 // Eq. 2 on many rows. bf16 rows with d = 64 or 128 go to the tensor-core kernel once there are enough of them to
 // pay for staging the split W per CTA; everything else runs on the CUDA-core kernel.
-int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments, cudaStream_t stream, bool* image_built = nullptr) {
+int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments, cudaStream_t stream, bool* image_built = nullptr,
+                bool pdl = false) {
   if (max_rows_per_segment <= 0 || segments <= 0) return HE_OK;
   const int Wd = words_of(job.b);
   const long long tiles = (max_rows_per_segment + kHashRows - 1) / kHashRows;
@@ -195,23 +206,25 @@ int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments
       HE_CUDA_CHECK(cudaGetLastError());
       if (image_built != nullptr) *image_built = true;
     }
-    if (Wd == 1) {
-      if (tma) {
-        if (int rc = set_smem(hash_rows_tc_kernel<1, true>, smem)) return rc;
-        hash_rows_tc_kernel<1, true><<<grid, kTcThreads, smem, stream>>>(job, total, tiles, tmap);
-      } else {
-        if (int rc = set_smem(hash_rows_tc_kernel<1, false>, smem)) return rc;
-        hash_rows_tc_kernel<1, false><<<grid, kTcThreads, smem, stream>>>(job, total, tiles, tmap);
-      }
-    } else {
-      if (tma) {
-        if (int rc = set_smem(hash_rows_tc_kernel<2, true>, smem)) return rc;
-        hash_rows_tc_kernel<2, true><<<grid, kTcThreads, smem, stream>>>(job, total, tiles, tmap);
-      } else {
-        if (int rc = set_smem(hash_rows_tc_kernel<2, false>, smem)) return rc;
-        hash_rows_tc_kernel<2, false><<<grid, kTcThreads, smem, stream>>>(job, total, tiles, tmap);
-      }
-    }
+    auto go = [&](auto kernel) -> int {
+      if (int rc = set_smem(kernel, smem)) return rc;
+      cudaLaunchConfig_t lc{};
+      lc.gridDim = dim3(grid);
+      lc.blockDim = dim3(kTcThreads);
+      lc.dynamicSmemBytes = smem;
+      lc.stream = stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      lc.attrs = attr;
+      lc.numAttrs = (pdl && pdl_enabled()) ? 1 : 0;
+      HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, kernel, job, total, tiles, tmap));
+      return HE_OK;
+    };
+    int rc;
+    if (Wd == 1) rc = tma ? go(hash_rows_tc_kernel<1, true>) : go(hash_rows_tc_kernel<1, false>);
+    else rc = tma ? go(hash_rows_tc_kernel<2, true>) : go(hash_rows_tc_kernel<2, false>);
+    if (rc) return rc;
     HE_CUDA_CHECK(cudaGetLastError());
     return HE_OK;
   }
@@ -227,16 +240,6 @@ int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments
   }
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
-}
-
-// Decode launches carry the programmatic-serialization attribute so that consecutive he_decode_step kernels of a
-// stream (or of a captured graph) overlap their launch latency; set HE_DISABLE_PDL=1 to launch them plainly.
-bool pdl_enabled() {
-  static const bool on = [] {
-    const char* e = getenv("HE_DISABLE_PDL");
-    return !(e && e[0] == '1');
-  }();
-  return on;
 }
 
 template <int WORDS, int GT, int NT, bool PRE>
@@ -429,7 +432,9 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
     job.x = k;
     job.out = cache->step_scratch + job.rows * Wd;
     job.rows = units_ll;
-    if (int rc = launch_hash(job, job.rows, 1, st, &image_built)) return rc;
+    // the key rows are hashed by a programmatically launched kernel: it needs nothing from the query-row kernel, so
+    // it may run beside it; it ends only after that kernel has ended, which is what the scan kernel's wait relies on
+    if (int rc = launch_hash(job, job.rows, 1, st, &image_built, true)) return rc;
     a.new_codes = cache->step_scratch;
   }
   if (cache->budget_host != nullptr && cfg->batch <= kMaxBudgetVals) {
