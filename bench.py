@@ -405,8 +405,8 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-folded", action="store_true", help="skip the secondary all-replicas-in-one-call decode figure")
     ap.add_argument("--e2e-steps", type=int, default=64)
-    ap.add_argument("--ref-seqs", type=int, default=2, help="sequences in the oracle's bounded sample")
-    ap.add_argument("--ref-decode-steps", type=int, default=64)
+    ap.add_argument("--ref-seqs", type=int, default=12, help="sequences in the oracle's bounded sample")
+    ap.add_argument("--ref-decode-steps", type=int, default=128)
     args = ap.parse_args()
     w = wl.CONFIGS[args.workload]
     if args.decode_steps is not None:
