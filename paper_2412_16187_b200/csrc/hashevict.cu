@@ -325,6 +325,7 @@ int launch_replay_reg(const ReplayArgs& a, long long units, cudaStream_t stream)
   if (c <= 256 * 8) return launch_replay_reg_one<WORDS, GT, 8, 256>(a, units, stream);
   if (c <= 256 * 16) return launch_replay_reg_one<WORDS, GT, 16, 256>(a, units, stream);
   if (c <= 512 * 16) return launch_replay_reg_one<WORDS, GT, 16, 512>(a, units, stream);
+  if (c <= 512 * 20) return launch_replay_reg_one<WORDS, GT, 20, 512>(a, units, stream);
   if (c <= 512 * 24) return launch_replay_reg_one<WORDS, GT, 24, 512>(a, units, stream);
   if (c <= 1024 * 16) return launch_replay_reg_one<WORDS, GT, 16, 1024>(a, units, stream);
   return launch_replay_smem<WORDS, GT>(a, units, stream);

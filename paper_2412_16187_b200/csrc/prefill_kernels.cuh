@@ -212,7 +212,7 @@ __device__ __forceinline__ int claim_unit(int32_t* sched, int lane) {
 // ------------------------------------------------------------------------------------------------ registers
 
 template <int WORDS, int GT, int SPT, int NT>
-__global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : 1)) prefill_replay_reg_kernel(const ReplayArgs a) {
+__global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : (NT <= 512 ? 2 : 1))) prefill_replay_reg_kernel(const ReplayArgs a) {
   using Stager = StepStager<WORDS, GT>;
   using Ctx = QueryCtx<WORDS, GT>;
   extern __shared__ __align__(16) int32_t pos_s[];  // [smem_slots]
