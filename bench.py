@@ -398,6 +398,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--replicas", type=int, default=None, help="independent layer replicas cycled by the decode loop")
     ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--hash-bits", type=int, default=None, help="override b (hash-dimension sweep of Section 4.7)")
     ap.add_argument("--batch", type=int, default=None, help="fewer sequences (profiling captures on a small case)")
     ap.add_argument("--prompt-factor", type=int, default=None, help="ragged workloads: prompt = factor x budget")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of a CUDA graph")
@@ -411,6 +412,8 @@ def main():
     w = wl.CONFIGS[args.workload]
     if args.decode_steps is not None:
         w = w.scaled(decode_steps=args.decode_steps)
+    if args.hash_bits is not None:
+        w = w.scaled(hash_bits=args.hash_bits)
     if args.batch is not None:
         w = w.scaled(batch=args.batch)
     if args.prompt_factor is not None:

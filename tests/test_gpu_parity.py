@@ -247,3 +247,13 @@ def test_large_batch_decode_hashes_new_rows_in_bulk():
     case.prefill()
     case.compare_state()
     case.decode(5)
+
+
+@pytest.mark.parametrize("b", [4, 8, 16, 24, 32, 64])
+def test_hash_dimension_sweep(b):
+    """The hash widths of the paper's ablation (Section 4.7, Table 9), 4 and 24 bits included: prefill then decode."""
+    w = PARITY_CASES["llama3_8b_gqa"].scaled(batch=2, prompt_len=640, budget=257, decode_steps=12, hash_bits=b)
+    case = Case(w)
+    case.prefill()
+    case.compare_state()
+    case.decode(12, check_every=4)
