@@ -49,6 +49,8 @@ def _load():
         lib.orc_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32]
         lib.orc_prefill_codes.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32]
         lib.orc_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32]
+        lib.orc_attend.argtypes = [vp, vp, vp, vp]
+        lib.orc_attend.restype = None
         for f in (lib.orc_hash, lib.orc_reset, lib.orc_step_codes, lib.orc_step, lib.orc_prefill_codes, lib.orc_prefill):
             f.restype = None
         _lib = lib
@@ -133,6 +135,13 @@ class OracleCache:
         _load().orc_step_codes(ctypes.byref(self._cfg), ctypes.byref(self._ca), _p(qcodes), _p(kcodes), _p(k), _p(v),
                                _p(victim), _p(evicted), self.threads)
         return victim, evicted
+
+    def attend(self, q):
+        """Eq. 1 over the compressed cache (Algorithm 1 line 6). q [B, H*G, d] -> fp64 [B, H*G, d]."""
+        assert q.flags.c_contiguous and q.shape == (self.B, self.H * self.G, self.d)
+        out = np.zeros((self.B, self.H * self.G, self.d), dtype=np.float64)
+        _load().orc_attend(ctypes.byref(self._cfg), ctypes.byref(self._ca), _p(q), _p(out))
+        return out
 
     @staticmethod
     def _strides(a):

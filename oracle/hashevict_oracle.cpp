@@ -13,6 +13,9 @@
 //                       Algorithm 1 runs for every later prompt token in order.
 //   orc_step*           "Decoding Stage": Algorithm 1 continued, one call per generated token.
 //
+//   orc_attend          Eq. 1 on the compressed cache (Algorithm 1 line 6): softmax(q K^T / sqrt(d)) V per query head,
+//                       over the valid slots of the head's KV unit, in fp64.
+//
 // Readings taken where the paper is silent (all restated in the design notes):
 //   * q_t is compared with the table BEFORE k_t is inserted (Algorithm 1 line 1).
 //   * arg-min ties go to the lowest slot index; the victim's slot is overwritten in place.
@@ -26,7 +29,8 @@
 // h(-x) = ~h(x), sgn(0) = 1; Eq. 3 (E[d_H]/b = theta/pi) at known angles; brute force of the
 // victim rule on tiny caches with unpacked bit arrays; the constant-budget and newest-resident
 // invariants; codes == hash(K) for every slot; prefill == reset + N steps; the storage closed
-// form of Section 4.7. Parity unpinned: none.
+// form of Section 4.7; orc_attend against a library softmax-attention in fp64, a single-slot cache, equal keys (mean
+// of V), invariance to the slot order. Parity unpinned: none.
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -279,3 +283,37 @@ extern "C" void orc_prefill(const orc_config* cfg, orc_cache* ca, const float* W
   orc_prefill_codes(cfg, ca, kc.data(), qc.data(), k, v, kv_strides, prompt_len, max_prompt_len, threads);
 }
 
+
+// Eq. 1 over the compressed cache (Algorithm 1 line 6): for every unit and each of its G query heads,
+//   out[g] = sum_j softmax_j( q_g . K_j / sqrt(d) ) V_j   over the valid slots j < fill.
+// q: [B, Hkv*G, d] in the cache dtype; out: [B, Hkv*G, d] fp64. A unit with no valid slot gives zeros.
+extern "C" void orc_attend(const orc_config* cfg, const orc_cache* ca, const void* q, double* out) {
+  const int d = cfg->head_dim, G = cfg->group_size, es = esize(cfg->dtype);
+  const int64_t units = (int64_t)cfg->batch * cfg->n_kv_heads, Cmax = cfg->max_budget;
+  for (int64_t u = 0; u < units; ++u) {
+    const int fill = ca->fill[u];
+    const char* K = (const char*)ca->k_cache + u * Cmax * d * es;
+    const char* V = (const char*)ca->v_cache + u * Cmax * d * es;
+    for (int g = 0; g < G; ++g) {
+      const char* qg = (const char*)q + (u * G + g) * d * es;
+      double* o = out + (u * G + g) * d;
+      for (int c = 0; c < d; ++c) o[c] = 0.0;
+      if (fill == 0) continue;
+      std::vector<double> sc(fill);
+      double mx = -INFINITY;
+      for (int j = 0; j < fill; ++j) {
+        double dot = 0.0;
+        for (int c = 0; c < d; ++c) dot += load_elem(qg, c, cfg->dtype) * load_elem(K, (int64_t)j * d + c, cfg->dtype);
+        sc[j] = dot / std::sqrt((double)d);
+        if (sc[j] > mx) mx = sc[j];
+      }
+      double den = 0.0;
+      for (int j = 0; j < fill; ++j) {
+        sc[j] = std::exp(sc[j] - mx);
+        den += sc[j];
+      }
+      for (int j = 0; j < fill; ++j)
+        for (int c = 0; c < d; ++c) o[c] += (sc[j] / den) * load_elem(V, (int64_t)j * d + c, cfg->dtype);
+    }
+  }
+}

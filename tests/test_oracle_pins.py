@@ -276,3 +276,44 @@ def test_hash_table_storage_closed_form():
     # the paper's 8- and 16-bit figures (20 MB, 40 MB) follow from the same b/8 bytes per slot
     slots = 80 * 8 * 8 * 4096
     assert [slots * b // 8 // 2 ** 20 for b in (8, 16, 32)] == [20, 40, 80]
+
+
+# ---------------------------------------------------------------- Eq. 1 on the compressed cache (Algorithm 1 line 6)
+
+def test_attend_matches_library_softmax_attention():
+    import torch
+
+    w, W, K, Q, V, oc = run_tiny(0, 0, 4, 16, C=16, N=40, T=0, dtype="bf16")
+    oc.prefill(W, Q, K, V, np.array([40, 11], dtype=np.int32))  # second sequence: 11 of 13 slots filled
+    q = np.ascontiguousarray(Q[:, :, 5])
+    out = oc.attend(q)
+    Kc, Vc, qd = (torch.from_numpy(wl.as_f64(w, a)) for a in (oc.k_cache, oc.v_cache, q))
+    for s in range(2):
+        for h in range(w.n_kv_heads):
+            f = int(oc.fill[s, h])
+            for g in range(4):
+                qq = qd[s, h * 4 + g]
+                p = torch.softmax((Kc[s, h, :f] @ qq) / np.sqrt(w.head_dim), dim=0)  # library softmax, fp64
+                np.testing.assert_allclose(out[s, h * 4 + g], (p[:, None] * Vc[s, h, :f]).sum(0).numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_attend_special_cases():
+    d = 16
+    oc = oracle.OracleCache(1, 1, 2, d, 8, 8, [8], "f32")
+    rng = np.random.default_rng(5)
+    q = rng.standard_normal((1, 2, d)).astype(np.float32)
+    assert not oc.attend(q).any()  # empty cache
+    oc.fill[:] = 1
+    oc.k_cache[0, 0, 0] = rng.standard_normal(d)
+    oc.v_cache[0, 0, 0] = np.arange(d)
+    np.testing.assert_allclose(oc.attend(q)[0, 1], np.arange(d), rtol=1e-15)  # one slot: its V row, whatever q is
+    oc.fill[:] = 5
+    oc.k_cache[0, 0, :5] = oc.k_cache[0, 0, 0]  # equal keys: uniform weights, the mean of V
+    oc.v_cache[0, 0, :5] = rng.standard_normal((5, d))
+    np.testing.assert_allclose(oc.attend(q)[0, 0], oc.v_cache[0, 0, :5].astype(np.float64).mean(0), rtol=1e-12, atol=1e-12)
+    oc.k_cache[0, 0, :5] = rng.standard_normal((5, d))
+    a = oc.attend(q).copy()
+    perm = np.array([3, 1, 4, 0, 2])
+    oc.k_cache[0, 0, :5] = oc.k_cache[0, 0, perm]
+    oc.v_cache[0, 0, :5] = oc.v_cache[0, 0, perm]
+    np.testing.assert_allclose(oc.attend(q), a, rtol=1e-12, atol=1e-13)  # the slot order does not matter
