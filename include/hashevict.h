@@ -131,6 +131,16 @@ size_t he_step_scratch_bytes(const he_config* cfg);
 /* Scratch bytes he_prefill_compress needs for prompts of up to max_prompt_len tokens (0 on bad input). */
 size_t he_workspace_bytes(const he_config* cfg, int32_t max_prompt_len);
 
+/*
+ * he_attend - attention over the compressed cache, the step that follows the eviction (Algorithm 1 line 6, Eq. 1):
+ *   out[s, h*G + g, :] = sum_j softmax_j( q[s, h*G + g, :] . K[s, h, j, :] / sqrt(d) ) * V[s, h, j, :]
+ * over the valid slots j < fill of unit (s, h). q: [B, Hkv*G, d] in the dtype of cfg (contiguous); out: [B, Hkv*G, d]
+ * fp32. Products of bf16 inputs are exact; sums and the softmax are carried in fp32 (exp2 of scaled scores, running
+ * maximum), so results agree with exact arithmetic to about 1e-5 of the largest |V| entry. A unit without valid
+ * slots gives zeros. The cache is only read.
+ */
+int he_attend(const he_config* cfg, const he_cache* cache, const void* q, float* out, void* stream);
+
 /* he_reset - empty every unit: fill = 0, next_pos = 0, pos = -1, codes = 0, scores = 0. K/V are left as they are. */
 int he_reset(const he_config* cfg, const he_cache* cache, void* stream);
 

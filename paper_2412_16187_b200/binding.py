@@ -36,7 +36,7 @@ class he_cache(ctypes.Structure):
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
     "he_decode_staging_bytes", "he_decode_step_host", "he_prefill_staging_bytes", "he_prefill_compress_host",
-    "he_prefill_compress_noalloc", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
+    "he_prefill_compress_noalloc", "he_attend", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
 )
 
 _lib = None
@@ -67,6 +67,8 @@ def lib():
     L.he_prefill_staging_bytes.restype = sz
     L.he_prefill_compress_host.argtypes = [cfgp, cap, vp, vp, vp, vp, i32, vp, vp, sz, vp]
     L.he_prefill_compress_noalloc.argtypes = [cfgp, cap, vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), vp, i32, vp]
+    L.he_attend.argtypes = [cfgp, cap, vp, vp, vp]
+    L.he_attend.restype = ctypes.c_int
     L.he_step_scratch_bytes.argtypes = [cfgp]
     L.he_step_scratch_bytes.restype = sz
     L.he_device_error_count.argtypes = []
@@ -171,6 +173,13 @@ class HashEvictCache:
         _check(lib().he_decode_step(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q), _ptr(k), _ptr(v),
                                     _ptr(victim_out), _ptr(evicted_pos_out), _ptr(qcodes_out), _stream(stream)))
         return victim_out
+
+    def attend(self, q, out=None, stream=None):
+        """he_attend: softmax(q K^T / sqrt(d)) V over the valid slots (Eq. 1). q [B, H*G, d] -> fp32 [B, H*G, d]."""
+        if out is None:
+            out = torch.empty((self.B, self.H * self.G, self.d), dtype=torch.float32, device=self.k_cache.device)
+        _check(lib().he_attend(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q), _ptr(out), _stream(stream)))
+        return out
 
     def workspace(self, max_prompt_len):
         need = workspace_bytes(self.cfg, max_prompt_len)

@@ -18,6 +18,7 @@
 #include <mutex>
 #include <utility>
 
+#include "attend_kernels.cuh"
 #include "common.cuh"
 #include "decode_kernels.cuh"
 #include "hash_kernels.cuh"
@@ -554,6 +555,46 @@ int he_prefill_compress_noalloc(const he_config* cfg, const he_cache* cache, con
   }
   return he_prefill_compress(cfg, cache, q, k, v, q_strides, kv_strides, prompt_len, max_prompt_len, scratch,
                              HE_NOALLOC_SCRATCH_BYTES, stream);
+}
+
+int he_attend(const he_config* cfg, const he_cache* cache, const void* q, float* out, void* stream) {
+  if (int rc = check_config(cfg, true)) return rc;
+  if (int rc = check_cache(cache)) return rc;
+  if (!q || !out || !aligned16(q) || !aligned16(out)) return fail(HE_ERR_INVALID_ARG, "q or out is null or not 16-byte aligned");
+  if (cfg->batch > 65535) return fail(HE_ERR_UNSUPPORTED, "batch %d > 65535 in one call", cfg->batch);
+  AttendArgs a{*cfg, *cache, q, out};
+  const dim3 grid((unsigned)cfg->n_kv_heads, (unsigned)cfg->batch);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int G = cfg->group_size, d = cfg->head_dim;
+  if (cfg->dtype == HE_DTYPE_BF16 && d == 128 && getenv("HE_DISABLE_ATTEND_MMA") == nullptr) {
+    // Cluster size: the largest power of two (<= 8) that keeps the grid within one CTA per SM.
+    const long long units = (long long)cfg->batch * cfg->n_kv_heads;
+    int sms = 0;
+    if (int rc = sm_count(&sms)) return rc;
+    int S = 1;
+    while (S < 8 && units * (S * 2) <= sms) S *= 2;
+    const size_t smem = (size_t)(kAttendWarps + 1) * G * (d + 2) * sizeof(float);
+    if (int rc = set_smem(attend_bf16_kernel, smem)) return rc;
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((unsigned)(cfg->n_kv_heads * S), (unsigned)cfg->batch);
+    lc.blockDim = dim3(kAttendThreads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)S;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, attend_bf16_kernel, a, S));
+  } else {
+    const size_t smem = ((size_t)G * d + (size_t)kAttendWarps * G * (d + 2)) * sizeof(float);
+    if (int rc = set_smem(attend_generic_kernel, smem)) return rc;
+    attend_generic_kernel<<<grid, kAttendThreads, smem, st>>>(a);
+  }
+  HE_CUDA_CHECK(cudaGetLastError());
+  return HE_OK;
 }
 
 int he_reset(const he_config* cfg, const he_cache* cache, void* stream) {
