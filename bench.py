@@ -375,6 +375,30 @@ def run_ours(args, w):
                                  "achieved_gbs": fbytes / us / 1e3, "frac": fbytes / us / 1e3 / peak}
         del big
 
+    if rank == 0 and not args.skip_attend:
+        # ---- secondary figure: Eq. 1 over the compressed caches the steps above left behind (Algorithm 1 line 6),
+        # one he_attend call per layer replica, rotating over the replicas so that K/V come from HBM, not L2
+        aq = gq[T - 1]
+        aout = torch.empty((B, H * G, d), dtype=torch.float32, device="cuda")
+        reps = max(1, int(np.ceil(64 / R)))
+        with torch.cuda.stream(stream):
+            for c in caches[:3]:
+                c.attend(aq, aout, stream=stream)
+            a0, a1 = ev(), ev()
+            a0.record(stream)
+            for _ in range(reps):
+                for c in caches:
+                    c.attend(aq, aout, stream=stream)
+            a1.record(stream)
+        torch.cuda.synchronize()
+        us = a0.elapsed_time(a1) * 1e3 / (reps * R)
+        esz = 2 if w.dtype == "bf16" else 4
+        abytes = float(caches[0].fill.sum().item()) * 2 * d * esz + B * H * G * d * (esz + 4)
+        line["attend"] = {"what": "he_attend: softmax(q K^T / sqrt(d)) V over the valid slots of every unit, one call per replica",
+                          "us_per_call": us, "bound": "hbm", "achieved": abytes / us / 1e3, "peak": peak, "unit": "GB/s",
+                          "frac": abytes / us / 1e3 / peak, "algorithmic_bytes_per_call": abytes,
+                          "kv_bytes_all_replicas": abytes * R}
+
     if rank == 0:
         line["clocks"] = clocks
         if not args.skip_cpu_baseline and world == 1:
@@ -404,6 +428,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of a CUDA graph")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-attend", action="store_true", help="skip the he_attend figure")
     ap.add_argument("--skip-folded", action="store_true", help="skip the secondary all-replicas-in-one-call decode figure")
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--ref-seqs", type=int, default=12, help="sequences in the oracle's bounded sample")
