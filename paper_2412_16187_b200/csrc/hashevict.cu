@@ -25,6 +25,7 @@
 #include "hash_tc_kernels.cuh"
 #include "hashevict.h"
 #include "prefill_kernels.cuh"
+#include "prefill_tc_kernels.cuh"
 
 using namespace he;
 
@@ -332,8 +333,34 @@ int launch_replay_reg(const ReplayArgs& a, long long units, cudaStream_t stream)
   return launch_replay_smem<WORDS, GT>(a, units, stream);
 }
 
+// Tensor-core replay: one persistent CTA per SM. Used when the whole table of a unit fits its shared-memory layout
+// (budgets up to 4096 slots) and no protected window is set.
+template <int WORDS>
+int launch_replay_tc(const ReplayArgs& a0, long long units, cudaStream_t stream) {
+  ReplayArgs a = a0;
+  a.smem_slots = (a.cfg.max_budget + kRtTile - 1) / kRtTile * kRtTile;
+  const size_t smem = rt_layout(WORDS, a.smem_slots, a.cfg.group_size).total;
+  if (int rc = set_smem(prefill_replay_tc_kernel<WORDS>, smem)) return rc;
+  int sms = 0;
+  if (int rc = sm_count(&sms)) return rc;
+  const int nbins = sms < kMaxBins ? sms : kMaxBins;
+  prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched);
+  HE_CUDA_CHECK(cudaGetLastError());
+  const long long grid = units < sms ? units : sms;
+  prefill_replay_tc_kernel<WORDS><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);
+  HE_CUDA_CHECK(cudaGetLastError());
+  return HE_OK;
+}
+
+bool tc_replay_enabled() {
+  const char* e = getenv("HE_TC_REPLAY");
+  return tc_enabled() && e && e[0] == '1';
+}
+
 template <int WORDS>
 int launch_replay(const ReplayArgs& a, long long units, cudaStream_t stream) {
+  if (tc_replay_enabled() && a.cfg.max_budget <= kRtMaxSlots && a.cfg.n_sink == 0 && a.cfg.n_recent == 0)
+    return launch_replay_tc<WORDS>(a, units, stream);
   switch (a.cfg.group_size) {
     case 1: return launch_replay_reg<WORDS, 1>(a, units, stream);
     case 4: return launch_replay_reg<WORDS, 4>(a, units, stream);

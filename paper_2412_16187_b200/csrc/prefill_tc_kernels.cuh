@@ -1,0 +1,507 @@
+// he_prefill_compress, phase 2 on the tensor cores: the sequential replay of Algorithm 1 over the prompt ("Prompt
+// Encoding Stage" of Section 3) with the Hamming distances of Eq. 5 taken 128 steps at a time as a dense product.
+//
+// Why this is a contraction. With codes read as +-1 vectors s, the group distance of slot j at step t is
+//   D(j, t) = sum_g popc(h_j xor h(q_{t,g})) = (G * K - <s_j, u_t>) / 2,   u_t = sum_g s(q_{t,g})  (entries in -G..G),
+// so the distances of all slots to a block of steps are one [steps x K] * [K x slots] product of small integers,
+// exact in bf16 operands and fp32 accumulation. Three more columns of the contraction turn the accumulator into
+// the arg-max key of Eq. 6 itself:  key(j, t) = D * 2^14 + (16383 - j)  (largest distance first, lowest slot on
+// ties): A = [-2^13 u_t | 128 | 1 | G K 2^13], B = [s_j | idx_j >> 7 | idx_j & 127 | 1], idx_j = 16383 - j. Every
+// partial sum is an integer below 2^24, so the result does not depend on the order of accumulation.
+//
+// What stays sequential. Step t must see the table as steps < t left it. A block of 128 steps is multiplied
+// against the table as it stood at the start of the block ("base" slots), and one more tile holds the distances
+// of the block's own 128 keys to the block's queries ("new" entries). A single warp then walks the block's steps
+// in order: the step's best base slot comes from per-tile maxima that the tensor-memory readers left in shared
+// memory, its best new entry from the extra tile, and a slot that an earlier step of the block has already evicted
+// is recognised by an owner table; only then is that tile's maximum recomputed for this step with popcounts. If
+// a block meets many such repairs it is cut short and the next block starts from the updated table, which bounds
+// the cost on adversarial data. The result is bit for bit that of the step-by-step scan.
+//
+// One persistent CTA per SM (units claimed from the same schedule as the register kernel), 416 threads:
+//   warps 0-3  read accumulators from tensor memory (one step per thread), reduce each 128-slot tile to its maximum
+//              key; warp 0 is also the resolver that walks the steps of a block
+//   warps 4-11 expand packed codes into +-1 bf16 operand tiles (K-major, 128-byte swizzle), one slot per thread,
+//              four warps per operand stage
+//   warp 12    one thread issues the tcgen05.mma instructions (M = 128 steps, N = 128 slots, K = 16) and commits
+// Every wait on an mbarrier is bounded; on a time-out the CTA raises a flag, leaves its loops through the same
+// barriers as usual, releases tensor memory and returns, and the device error counter is incremented.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "hash_tc_kernels.cuh"
+#include "prefill_kernels.cuh"
+
+namespace he {
+
+constexpr int kRtThreads = 416;
+constexpr int kRtMmaWarp = kRtThreads / 32 - 1;
+constexpr int kRtRows = 128;       // steps per block = MMA M
+constexpr int kRtTile = 128;       // slots per tile = MMA N
+constexpr int kRtMaxSlots = 4096;  // 32 tiles: one tile maximum per resolver lane
+constexpr int kRtMPitch = 33;      // words per row of the tile-maximum table (odd: conflict-free column writes)
+constexpr int kRtKeyShift = 14;
+constexpr int kRtIdxMask = (1 << kRtKeyShift) - 1;
+constexpr int kRtStaleLimit = 64;  // repairs after which a block is cut short
+constexpr int kRtAtomBytes = kRtRows * 128;  // one 64-column K-major swizzle atom of a 128-row operand tile
+
+// Byte offsets of the kernel's dynamic shared memory (after rounding its base up to 1024 bytes).
+struct RtLayout {
+  uint32_t a, b, codes, pos, owner, m, rb, dn, qraw, kraw, total;
+};
+__host__ __device__ inline RtLayout rt_layout(int words, int slots, int G) {
+  RtLayout L;
+  const uint32_t atoms = words == 2 ? 2u : 1u;
+  uint32_t o = 0;
+  L.a = o, o += atoms * kRtAtomBytes;
+  L.b = o, o += 2u * atoms * kRtAtomBytes;
+  L.codes = o, o += (uint32_t)slots * words * 4u;
+  L.pos = o, o += (uint32_t)slots * 4u;
+  L.owner = o, o += (uint32_t)slots * 2u;
+  L.m = o, o += kRtRows * kRtMPitch * 4u;
+  L.rb = o, o += kRtRows * 4u;
+  L.dn = o, o += kRtRows * kRtRows * 2u;
+  L.qraw = o, o += 2u * kRtRows * G * words * 4u;  // two buffers: this block's codes and the next block's
+  L.kraw = o, o += 2u * kRtRows * words * 4u;
+  L.total = o + 1024u;
+  return L;
+}
+
+// Byte offset of 16-byte chunk `chunk` (0..7) of row `row` inside one swizzle atom.
+__device__ __forceinline__ uint32_t rt_swz(int row, int chunk) {
+  return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4));
+}
+
+// bf16 bit pattern of a small non-negative integer (< 256: exact).
+__device__ __forceinline__ uint32_t rt_bf16_of_int(int x) { return __float_as_uint((float)x) >> 16; }
+
+// Eight code bits (bits 8c .. 8c+7 of the code) as eight +-1 bf16 values: bit set -> +1 (0x3F80), clear -> -1 (0xBF80).
+__device__ __forceinline__ uint4 rt_expand8(uint32_t byte) {
+  const uint32_t x = ~byte;
+  uint4 v;
+  v.x = 0x3F803F80u | ((x << 15) & 0x8000u) | ((x << 30) & 0x80000000u);
+  v.y = 0x3F803F80u | ((x << 13) & 0x8000u) | ((x << 28) & 0x80000000u);
+  v.z = 0x3F803F80u | ((x << 11) & 0x8000u) | ((x << 26) & 0x80000000u);
+  v.w = 0x3F803F80u | ((x << 9) & 0x8000u) | ((x << 24) & 0x80000000u);
+  return v;
+}
+
+// Group distance of Eq. 5 straight from the packed words (used for the few slots the resolver looks at itself).
+template <int WORDS>
+__device__ __forceinline__ int rt_dist(const uint32_t* h, const uint32_t* q, int G) {
+  int D = 0;
+  for (int g = 0; g < G; ++g) {
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w) D += __popc(h[w] ^ q[g * WORDS + w]);
+  }
+  return D;
+}
+
+template <int WORDS>
+__global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const ReplayArgs a) {
+  constexpr int ATOMS = WORDS == 2 ? 2 : 1;
+  constexpr int KB = 32 * WORDS;             // code columns of the contraction
+  constexpr int KSTEPS = (KB + 16) / 16;     // MMA instructions per tile (the last one holds the three key columns)
+  constexpr int XATOM = KB / 64, XCHUNK = (KB % 64) / 8;  // where the key columns start
+  constexpr int NT = kRtThreads;
+  extern __shared__ unsigned char rt_smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[8];
+  __shared__ uint32_t tmem_base_s;
+  __shared__ volatile int abort_flag;
+  __shared__ int s_unit, s_done;
+  // four code bits -> four bf16 values: operand B takes +-1 (bit set: +1), operand A -+2^13 (bit set: -2^13)
+  __shared__ uint2 s_lut_a[16], s_lut_b[16];
+
+  const he_config& cfg = a.cfg;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int G = cfg.group_size;
+  const long long Cmax = cfg.max_budget;
+  const bool write_scores = (cfg.flags & HE_FLAG_WRITE_SCORES) != 0;
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(rt_smem_raw) + 1023) & ~(uintptr_t)1023);
+  const RtLayout L = rt_layout(WORDS, a.smem_slots, G);
+  unsigned char* As = smem + L.a;
+  unsigned char* Bs = smem + L.b;
+  uint32_t* codes_t = reinterpret_cast<uint32_t*>(smem + L.codes);
+  int32_t* pos_t = reinterpret_cast<int32_t*>(smem + L.pos);
+  int16_t* owner = reinterpret_cast<int16_t*>(smem + L.owner);
+  int32_t* Mx = reinterpret_cast<int32_t*>(smem + L.m);
+  int32_t* RB = reinterpret_cast<int32_t*>(smem + L.rb);
+  uint16_t* Dn = reinterpret_cast<uint16_t*>(smem + L.dn);
+  uint32_t* qraw = reinterpret_cast<uint32_t*>(smem + L.qraw);
+  uint32_t* kraw = reinterpret_cast<uint32_t*>(smem + L.kraw);
+
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };          // expanders -> MMA: operand stage s is written
+  auto empty_bar = [&](int s) { return bar0 + 8u * (2 + s); };   // MMA -> expanders: stage s has been read
+  auto tfull_bar = [&](int x) { return bar0 + 8u * (4 + x); };   // MMA -> readers: accumulator x is complete
+  auto tempty_bar = [&](int x) { return bar0 + 8u * (6 + x); };  // readers -> MMA: accumulator x is drained
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(full_bar(s), 128);
+      mbar_init(empty_bar(s), 1);
+      mbar_init(tfull_bar(s), 1);
+      mbar_init(tempty_bar(s), 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (tid < 16) {
+    auto pick = [&](int bit, uint32_t set, uint32_t clear) { return ((tid >> bit) & 1) ? set : clear; };
+    s_lut_b[tid] = make_uint2(pick(0, 0x3F80u, 0xBF80u) | (pick(1, 0x3F80u, 0xBF80u) << 16),
+                              pick(2, 0x3F80u, 0xBF80u) | (pick(3, 0x3F80u, 0xBF80u) << 16));
+    s_lut_a[tid] = make_uint2(pick(0, 0xC600u, 0x4600u) | (pick(1, 0xC600u, 0x4600u) << 16),
+                              pick(2, 0xC600u, 0x4600u) | (pick(3, 0xC600u, 0x4600u) << 16));
+  }
+  if (warp == kRtMmaWarp) {  // two accumulators of 128 columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2 * kRtTile)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+  const uint32_t idesc = (1u << 4) /* fp32 accumulate */ | (1u << 7) /* A bf16 */ | (1u << 10) /* B bf16 */ |
+                         ((uint32_t)(kRtTile >> 3) << 17) | ((uint32_t)(kRtRows >> 4) << 24);
+  const uint32_t kconst_bits = __float_as_uint((float)(G * KB / 2) * 16384.f) >> 16;  // exact: G K / 2 <= 256
+  int it = 0;  // operand tiles processed so far; every role counts the same sequence
+
+  for (;;) {
+    if (warp == 0) {
+      const int u = claim_unit(a.sched, lane);
+      if (lane == 0) s_unit = u;
+    }
+    __syncthreads();
+    const long long unit = s_unit;
+    if (unit < 0) break;
+    const int s = (int)(unit / cfg.n_kv_heads);
+    const int C = min(a.ca.budget[s], (int)Cmax);
+    const int N = a.prompt_len[s];
+    const int fill0 = N < C ? N : C;
+    const uint32_t* kc_u = a.kcodes + unit * a.Nmax * WORDS;
+    const uint32_t* qc_u = a.qcodes + unit * a.Nmax * G * WORDS;
+    float* sc = a.ca.scores + unit * Cmax;
+    const int nbase = (C + kRtTile - 1) / kRtTile;
+    // the first C tokens fill the cache in order
+    for (int j = tid; j < a.smem_slots; j += NT) {
+#pragma unroll
+      for (int w = 0; w < WORDS; ++w) codes_t[j * WORDS + w] = j < fill0 ? __ldg(kc_u + (long long)j * WORDS + w) : 0u;
+      pos_t[j] = j < fill0 ? j : -1;
+    }
+    __syncthreads();
+    bool aborted = false;
+    const int GW = G * WORDS;
+    // The block's query and key codes into buffer `buf` (rows past the prompt are zero).
+    auto stage_codes = [&](int buf, int tb, int nrows, int first, int nthreads) {
+      uint32_t* qd = qraw + buf * kRtRows * GW;
+      uint32_t* kd = kraw + buf * kRtRows * WORDS;
+      for (int i = first; i < kRtRows * GW; i += nthreads) qd[i] = i < nrows * GW ? __ldg(qc_u + (long long)tb * GW + i) : 0u;
+      for (int i = first; i < kRtRows * WORDS; i += nthreads) kd[i] = i < nrows * WORDS ? __ldg(kc_u + (long long)tb * WORDS + i) : 0u;
+    };
+    // Operand A from buffer `buf`: row r = step r of the block, columns -2^13 u_t (sum over the group's heads of
+    // -+2^13 per bit, exact in packed bf16 adds), then the three key columns 128, 1, G K 2^13.
+    auto build_a = [&](int buf, int nrows, int first, int nthreads) {
+      const uint32_t* qd = qraw + buf * kRtRows * GW;
+      for (int item = first; item < kRtRows * (KB / 8 + 1); item += nthreads) {
+        const int r = item / (KB / 8 + 1), c = item % (KB / 8 + 1);
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (c < KB / 8) {
+          if (r < nrows) {
+            const int w = c >> 2, sh = (c & 3) * 8;
+            __nv_bfloat162 s0 = __float2bfloat162_rn(0.f), s1 = s0, s2 = s0, s3 = s0;
+            for (int g = 0; g < G; ++g) {
+              const uint32_t byte = qd[r * GW + g * WORDS + w] >> sh;
+              const uint2 lo = s_lut_a[byte & 15u], hi = s_lut_a[(byte >> 4) & 15u];
+              s0 = __hadd2(s0, *reinterpret_cast<const __nv_bfloat162*>(&lo.x));
+              s1 = __hadd2(s1, *reinterpret_cast<const __nv_bfloat162*>(&lo.y));
+              s2 = __hadd2(s2, *reinterpret_cast<const __nv_bfloat162*>(&hi.x));
+              s3 = __hadd2(s3, *reinterpret_cast<const __nv_bfloat162*>(&hi.y));
+            }
+            v = make_uint4(*reinterpret_cast<uint32_t*>(&s0), *reinterpret_cast<uint32_t*>(&s1),
+                           *reinterpret_cast<uint32_t*>(&s2), *reinterpret_cast<uint32_t*>(&s3));
+          }
+          *reinterpret_cast<uint4*>(As + (c >> 3) * kRtAtomBytes + rt_swz(r, c & 7)) = v;
+        } else {
+          if (r < nrows) v = make_uint4(0x4300u | (0x3F80u << 16), kconst_bits, 0u, 0u);
+          *reinterpret_cast<uint4*>(As + XATOM * kRtAtomBytes + rt_swz(r, XCHUNK)) = v;
+          *reinterpret_cast<uint4*>(As + XATOM * kRtAtomBytes + rt_swz(r, XCHUNK + 1)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+    };
+    int t0 = C, cur = 0;
+    bool staged = false;  // buffer `cur` and operand A already hold the block that starts at t0
+    while (t0 < N) {
+      const int rows = (N - t0) < kRtRows ? (N - t0) : kRtRows;
+      if (!staged) {  // first block of a unit, or the block before was cut short
+        stage_codes(cur, t0, rows, tid, NT);
+        __syncthreads();
+        build_a(cur, rows, tid, NT);
+        fence_proxy_async();
+        __syncthreads();
+      }
+      const uint32_t* qb = qraw + cur * kRtRows * GW;
+      const uint32_t* kb_codes = kraw + cur * kRtRows * WORDS;
+      // ---- tiles 0 .. nbase-1: base slots; tile nbase: the block's own keys
+      const int ntile = nbase + 1;
+      if (warp >= 4 && warp < kRtMmaWarp) {
+        // owner table cleared (-1: the slot still holds its base token); read only by the resolver
+        for (int i = tid - 128; i < a.smem_slots / 2; i += 256) reinterpret_cast<uint32_t*>(owner)[i] = 0xFFFFFFFFu;
+        // two groups of four warps, one per operand stage: group g expands the tiles that go to stage g
+        const int x = (tid - 128) & 127, grp = (tid - 128) >> 7;  // x: this thread's row of the tile
+        for (int i = 0; i < ntile; ++i) {
+          const int n = it + i, st = n & 1;
+          if (st != grp) continue;
+          if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(st), ((n >> 1) & 1) ^ 1, &abort_flag))) break;
+          unsigned char* bt = Bs + st * ATOMS * kRtAtomBytes;
+          uint32_t h[WORDS];
+          bool valid;
+          int idx;
+          if (i < nbase) {
+            const int j = i * kRtTile + x;
+            valid = j < C;
+            idx = kRtIdxMask - j;
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) h[w] = codes_t[j * WORDS + w];
+          } else {  // the block's own keys: plain distances, no index term
+            valid = x < rows;
+            idx = 0;
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) h[w] = kb_codes[x * WORDS + w];
+          }
+          const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+          for (int c = 0; c < KB / 8; ++c) {
+            const uint32_t byte = h[c >> 2] >> ((c & 3) * 8);
+            const uint2 lo = s_lut_b[byte & 15u], hi = s_lut_b[(byte >> 4) & 15u];
+            *reinterpret_cast<uint4*>(bt + (c >> 3) * kRtAtomBytes + rt_swz(x, c & 7)) = valid ? make_uint4(lo.x, lo.y, hi.x, hi.y) : zero;
+          }
+          *reinterpret_cast<uint4*>(bt + XATOM * kRtAtomBytes + rt_swz(x, XCHUNK)) =
+              valid ? make_uint4(rt_bf16_of_int(idx >> 7) | (rt_bf16_of_int(idx & 127) << 16), 0x3F80u, 0u, 0u) : zero;
+          *reinterpret_cast<uint4*>(bt + XATOM * kRtAtomBytes + rt_swz(x, XCHUNK + 1)) = zero;
+          fence_proxy_async();
+          mbar_arrive(full_bar(st));
+        }
+      } else if (warp == kRtMmaWarp) {
+        if (lane == 0) {
+          const uint64_t a_desc0 = umma_desc_k128(smem_u32(As));
+          for (int i = 0; i < ntile; ++i) {
+            const int n = it + i, st = n & 1;
+            if (!mbar_wait(tempty_bar(st), ((n >> 1) & 1) ^ 1, &abort_flag)) break;  // readers have drained this accumulator
+            if (!mbar_wait(full_bar(st), (n >> 1) & 1, &abort_flag)) break;
+            tc_fence_after();
+            const uint64_t b_desc0 = umma_desc_k128(smem_u32(Bs + st * ATOMS * kRtAtomBytes));
+            const uint32_t d_tmem = tmem_base + (uint32_t)(st * kRtTile);
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+              const uint32_t off = (uint32_t)(((ks * 16) / 64) * kRtAtomBytes + ((ks * 16) % 64) * 2);
+              tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)(off >> 4), b_desc0 + (uint64_t)(off >> 4), idesc, ks > 0);
+            }
+            tc_commit(empty_bar(st));   // the operand stage may be rewritten once these MMAs have read it
+            tc_commit(tfull_bar(st));   // and the accumulator is complete
+          }
+        }
+      } else {
+        bool ok = true;
+        for (int i = 0; i < ntile && ok; ++i) {
+          const int n = it + i, st = n & 1;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(st), (n >> 1) & 1, &abort_flag));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(st * kRtTile);
+          if (i < nbase) {  // the tile's largest key for this step (keys are non-negative floats: compare the bits)
+            uint32_t mx = 0u;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              uint32_t v[32];
+              tc_ld32(taddr + c * 32, v);
+              tc_wait_ld();
+#pragma unroll
+              for (int k = 0; k < 32; ++k) mx = max(mx, v[k]);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(st));
+            Mx[tid * kRtMPitch + i] = __float2int_rn(__uint_as_float(mx));
+          } else {  // distances of the block's keys: key / 2^14, kept as 16-bit integers
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              uint32_t v[32];
+              tc_ld32(taddr + c * 32, v);
+              tc_wait_ld();
+              uint32_t pk[16];
+#pragma unroll
+              for (int k = 0; k < 16; ++k)
+                pk[k] = (uint32_t)__float2int_rn(__uint_as_float(v[2 * k]) * (1.f / 16384.f)) |
+                        ((uint32_t)__float2int_rn(__uint_as_float(v[2 * k + 1]) * (1.f / 16384.f)) << 16);
+              uint4* dst = reinterpret_cast<uint4*>(Dn + tid * kRtRows + c * 32);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) dst[k] = make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(st));
+          }
+        }
+        if (ok) {
+          int rb = 0;
+          for (int i = 0; i < nbase; ++i) rb = max(rb, Mx[tid * kRtMPitch + i]);
+          RB[tid] = rb;
+        }
+      }
+      it += ntile;
+      tc_fence_before();
+      __syncthreads();
+      tc_fence_after();
+      if (abort_flag) {
+        aborted = true;
+        break;
+      }
+      // ---- the block's steps in order (warp 0); meanwhile the other warps prepare the next block's codes and
+      // operand A, which do not depend on this block's outcome (only on where the next block starts)
+      const int tn = t0 + rows;
+      if (warp == 0) {
+        // Lane l keeps the block's new entries e = 4l .. 4l+3 as the index half of their keys (16383 - slot), or a
+        // large negative number while absent or evicted. Everything a step reads that does not depend on the step
+        // before it (its row of new-entry distances, its best base key and that slot's owner, its key code) is
+        // fetched one step ahead, so the chain from step to step is a few integer operations and one warp reduction.
+        // The two rare cases (a stale base maximum, the scoring pass of the prompt's last step) leave the hot loop,
+        // are dealt with outside it and re-enter at the same step: the loop body stays small for the compiler.
+        constexpr int kAbsent = -(1 << 30);
+        int vb0 = kAbsent, vb1 = kAbsent, vb2 = kAbsent, vb3 = kAbsent;
+        int done = rows, stale = 0;
+        uint2 dd = *reinterpret_cast<const uint2*>(Dn + 4 * lane);
+        int kb = RB[0];
+        int own_kb = -1;  // nothing has been evicted yet
+        uint32_t kc[WORDS];
+#pragma unroll
+        for (int w = 0; w < WORDS; ++w) kc[w] = kb_codes[w];
+        bool scored = !(write_scores && t0 + rows == N);  // only the prompt's last step stores Eq. 5 scores
+        int r = 0;
+        while (r < rows) {
+          int status = 0;
+          for (; r < rows; ++r) {
+            const int rn = r + 1 < rows ? r + 1 : r;  // the last step fetches its own row again (unused)
+            const uint2 dd_n = *reinterpret_cast<const uint2*>(Dn + rn * kRtRows + 4 * lane);
+            const int kb_n = RB[rn];
+            int own_n = owner[kRtIdxMask - (kb_n & kRtIdxMask)];
+            uint32_t kc_n[WORDS];
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) kc_n[w] = kb_codes[rn * WORDS + w];
+            // best new entry (inserted by an earlier step of this block and still resident)
+            const int k0 = (int)((dd.x & 0xFFFFu) << kRtKeyShift) + vb0;
+            const int k1 = (int)((dd.x >> 16) << kRtKeyShift) + vb1;
+            const int k2 = (int)((dd.y & 0xFFFFu) << kRtKeyShift) + vb2;
+            const int k3 = (int)((dd.y >> 16) << kRtKeyShift) + vb3;
+            const int kn = __reduce_max_sync(0xFFFFFFFFu, max(max(k0, k1), max(k2, k3)));
+            // best base slot: the tile maxima are upper bounds; one that points at an evicted slot needs a repair
+            if (kb > kn && own_kb >= 0) {
+              status = 1;
+              break;
+            }
+            if (!scored && r == rows - 1) {
+              status = 2;
+              break;
+            }
+            const int best = max(kb, kn);
+            const int slot = kRtIdxMask - (best & kRtIdxMask);
+            // a new entry that wins leaves: its lane recognises its own key (keys of resident entries are distinct,
+            // absent ones are negative); then this step's token enters as entry r
+            const bool mine = lane == (r >> 2);
+            const int sel = r & 3, nv = kRtIdxMask - slot;
+            vb0 = (mine && sel == 0) ? nv : (k0 == best ? kAbsent : vb0);
+            vb1 = (mine && sel == 1) ? nv : (k1 == best ? kAbsent : vb1);
+            vb2 = (mine && sel == 2) ? nv : (k2 == best ? kAbsent : vb2);
+            vb3 = (mine && sel == 3) ? nv : (k3 == best ? kAbsent : vb3);
+            // Algorithm 1 lines 2-5 on the table (K / V rows follow in the gather kernel). Every lane stores the same
+            // values to the same addresses: no divergent branch, and each lane later reads back its own stores.
+            owner[slot] = (int16_t)r;
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
+            pos_t[slot] = t0 + r;
+            if (slot == kRtIdxMask - (kb_n & kRtIdxMask)) own_n = r;  // the owner fetched ahead predates this step
+            dd = dd_n, kb = kb_n, own_kb = own_n;
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) kc[w] = kc_n[w];
+          }
+          if (status == 1) {
+            // Repair for step r: recompute the maximum of the tile the stale key came from, over the slots that
+            // still hold their base token, until the row's best base key is exact (or no longer matters). Each pass
+            // makes one tile exact, so nbase passes always suffice; the bound only guards against a corrupted table.
+            const uint32_t* qr = qb + r * GW;
+            const int k0 = (int)((dd.x & 0xFFFFu) << kRtKeyShift) + vb0;
+            const int k1 = (int)((dd.x >> 16) << kRtKeyShift) + vb1;
+            const int k2 = (int)((dd.y & 0xFFFFu) << kRtKeyShift) + vb2;
+            const int k3 = (int)((dd.y >> 16) << kRtKeyShift) + vb3;
+            const int kn = __reduce_max_sync(0xFFFFFFFFu, max(max(k0, k1), max(k2, k3)));
+            for (int pass = 0; pass <= nbase; ++pass) {
+              ++stale;
+              const int cb = (kRtIdxMask - (kb & kRtIdxMask)) / kRtTile;
+              int km = 0;
+#pragma unroll
+              for (int i = 0; i < kRtTile / 32; ++i) {
+                const int j = cb * kRtTile + lane + 32 * i;
+                if (j < C && owner[j] < 0) km = max(km, (rt_dist<WORDS>(codes_t + j * WORDS, qr, G) << kRtKeyShift) + (kRtIdxMask - j));
+              }
+              km = __reduce_max_sync(0xFFFFFFFFu, km);
+              Mx[r * kRtMPitch + cb] = km;  // same value from every lane
+              kb = __reduce_max_sync(0xFFFFFFFFu, lane < nbase ? Mx[r * kRtMPitch + lane] : 0);
+              if (kb <= kn || owner[kRtIdxMask - (kb & kRtIdxMask)] < 0) break;
+            }
+            own_kb = -1;  // exact for this step (or below the best new entry)
+            if (stale >= kRtStaleLimit && r + 1 < rows && scored) {  // many repairs: this block ends with step r
+              // finish step r here, then stop
+              const int best = max(kb, kn);
+              const int slot = kRtIdxMask - (best & kRtIdxMask);
+              owner[slot] = (int16_t)r;
+#pragma unroll
+              for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
+              pos_t[slot] = t0 + r;
+              done = r + 1;
+              break;
+            }
+          } else if (status == 2) {  // Eq. 5 for every slot as the prompt's last step sees the table
+            const uint32_t* qr = qb + r * GW;
+            for (int j = lane; j < C; j += 32) sc[j] = -(float)rt_dist<WORDS>(codes_t + j * WORDS, qr, G);
+            scored = true;
+          }
+        }
+        if (lane == 0) s_done = done;
+      } else if (tn < N) {
+        const int nrows = (N - tn) < kRtRows ? (N - tn) : kRtRows;
+        stage_codes(cur ^ 1, tn, nrows, tid - 32, NT - 32);
+        asm volatile("bar.sync 1, %0;" ::"n"(NT - 32) : "memory");
+        build_a(cur ^ 1, nrows, tid - 32, NT - 32);
+        fence_proxy_async();
+      }
+      __syncthreads();
+      staged = s_done == rows;  // a block that was cut short restarts from its first unprocessed step
+      t0 += s_done;
+      if (staged) cur ^= 1;
+    }
+    if (aborted) break;
+    // final state of the unit; everything beyond `fill` is reset
+    const bool scored = write_scores && N > C;
+    for (int j = tid; j < Cmax; j += NT) {
+      const bool valid = j < fill0;
+#pragma unroll
+      for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = valid ? codes_t[j * WORDS + w] : 0u;
+      a.ca.pos[unit * Cmax + j] = valid ? pos_t[j] : -1;
+      if (!(valid && scored)) sc[j] = 0.f;
+    }
+    if (tid == 0) {
+      a.ca.fill[unit] = fill0;
+      a.ca.next_pos[unit] = N;
+    }
+    __syncthreads();  // the tables and s_unit are reused by the next unit
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kRtMmaWarp) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kRtTile) : "memory");
+  }
+  if (tid == 0 && abort_flag) atomicAdd(&g_tc_error, 1);
+}
+
+}  // namespace he
