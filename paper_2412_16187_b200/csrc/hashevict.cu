@@ -352,14 +352,19 @@ int launch_replay_tc(const ReplayArgs& a0, long long units, cudaStream_t stream)
   return HE_OK;
 }
 
-bool tc_replay_enabled() {
+// HE_TC_REPLAY=0 keeps the replay on the CUDA-core kernels, =1 sends every eligible shape to the tensor-core kernel;
+// unset, the tensor-core kernel takes budgets from 512 slots up (below that a block of 128 steps no longer pays).
+int tc_replay_mode() {
   const char* e = getenv("HE_TC_REPLAY");
-  return tc_enabled() && e && e[0] == '1';
+  if (!tc_enabled() || (e && e[0] == '0')) return 0;
+  return (e && e[0] == '1') ? 2 : 1;
 }
 
 template <int WORDS>
 int launch_replay(const ReplayArgs& a, long long units, cudaStream_t stream) {
-  if (tc_replay_enabled() && a.cfg.max_budget <= kRtMaxSlots && a.cfg.n_sink == 0 && a.cfg.n_recent == 0)
+  const int mode = tc_replay_mode();
+  if (mode != 0 && a.cfg.max_budget <= kRtMaxSlots && (mode == 2 || a.cfg.max_budget >= 512) && a.cfg.n_sink == 0 &&
+      a.cfg.n_recent == 0)
     return launch_replay_tc<WORDS>(a, units, stream);
   switch (a.cfg.group_size) {
     case 1: return launch_replay_reg<WORDS, 1>(a, units, stream);

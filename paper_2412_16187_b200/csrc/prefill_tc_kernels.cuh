@@ -98,6 +98,7 @@ __device__ __forceinline__ int rt_dist(const uint32_t* h, const uint32_t* q, int
 }
 
 template <int WORDS>
+// 13 warps: one scheduler hosts four of them, so 128 registers per thread is the most its 16 K registers allow
 __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const ReplayArgs a) {
   constexpr int ATOMS = WORDS == 2 ? 2 : 1;
   constexpr int KB = 32 * WORDS;             // code columns of the contraction
@@ -269,15 +270,23 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             for (int w = 0; w < WORDS; ++w) h[w] = kb_codes[x * WORDS + w];
           }
           const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+          unsigned char* brow = bt + (x >> 3) * 1024 + (x & 7) * 128;  // this row inside each swizzle atom
+          const int xs = (x & 7) << 4;
+          if (valid) {
 #pragma unroll
-          for (int c = 0; c < KB / 8; ++c) {
-            const uint32_t byte = h[c >> 2] >> ((c & 3) * 8);
-            const uint2 lo = s_lut_b[byte & 15u], hi = s_lut_b[(byte >> 4) & 15u];
-            *reinterpret_cast<uint4*>(bt + (c >> 3) * kRtAtomBytes + rt_swz(x, c & 7)) = valid ? make_uint4(lo.x, lo.y, hi.x, hi.y) : zero;
+            for (int c = 0; c < KB / 8; ++c) {
+              const uint32_t byte = h[c >> 2] >> ((c & 3) * 8);
+              const uint2 lo = s_lut_b[byte & 15u], hi = s_lut_b[(byte >> 4) & 15u];
+              *reinterpret_cast<uint4*>(brow + (c >> 3) * kRtAtomBytes + (((c & 7) << 4) ^ xs)) = make_uint4(lo.x, lo.y, hi.x, hi.y);
+            }
+            *reinterpret_cast<uint4*>(brow + XATOM * kRtAtomBytes + ((XCHUNK << 4) ^ xs)) =
+                make_uint4(rt_bf16_of_int(idx >> 7) | (rt_bf16_of_int(idx & 127) << 16), 0x3F80u, 0u, 0u);
+          } else {  // a row past the budget (or past the block's steps): all zeros, its key is 0
+#pragma unroll
+            for (int c = 0; c < KB / 8; ++c) *reinterpret_cast<uint4*>(brow + (c >> 3) * kRtAtomBytes + (((c & 7) << 4) ^ xs)) = zero;
+            *reinterpret_cast<uint4*>(brow + XATOM * kRtAtomBytes + ((XCHUNK << 4) ^ xs)) = zero;
           }
-          *reinterpret_cast<uint4*>(bt + XATOM * kRtAtomBytes + rt_swz(x, XCHUNK)) =
-              valid ? make_uint4(rt_bf16_of_int(idx >> 7) | (rt_bf16_of_int(idx & 127) << 16), 0x3F80u, 0u, 0u) : zero;
-          *reinterpret_cast<uint4*>(bt + XATOM * kRtAtomBytes + rt_swz(x, XCHUNK + 1)) = zero;
+          *reinterpret_cast<uint4*>(brow + XATOM * kRtAtomBytes + (((XCHUNK + 1) << 4) ^ xs)) = zero;
           fence_proxy_async();
           mbar_arrive(full_bar(st));
         }
@@ -311,12 +320,13 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           if (i < nbase) {  // the tile's largest key for this step (keys are non-negative floats: compare the bits)
             uint32_t mx = 0u;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              uint32_t v[32];
-              tc_ld32(taddr + c * 32, v);
+            for (int c = 0; c < 4; c += 2) {  // two loads in flight per wait
+              uint32_t v0[32], v1[32];
+              tc_ld32(taddr + c * 32, v0);
+              tc_ld32(taddr + c * 32 + 32, v1);
               tc_wait_ld();
 #pragma unroll
-              for (int k = 0; k < 32; ++k) mx = max(mx, v[k]);
+              for (int k = 0; k < 32; ++k) mx = max(mx, max(v0[k], v1[k]));
             }
             tc_fence_before();
             __syncwarp();
@@ -427,7 +437,9 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             // Repair for step r: recompute the maximum of the tile the stale key came from, over the slots that
             // still hold their base token, until the row's best base key is exact (or no longer matters). Each pass
             // makes one tile exact, so nbase passes always suffice; the bound only guards against a corrupted table.
-            const uint32_t* qr = qb + r * GW;
+            uint32_t qw[kMaxGroup * WORDS];
+#pragma unroll
+            for (int i = 0; i < kMaxGroup * WORDS; ++i) qw[i] = i < GW ? qb[r * GW + i] : 0u;
             const int k0 = (int)((dd.x & 0xFFFFu) << kRtKeyShift) + vb0;
             const int k1 = (int)((dd.x >> 16) << kRtKeyShift) + vb1;
             const int k2 = (int)((dd.y & 0xFFFFu) << kRtKeyShift) + vb2;
@@ -436,11 +448,28 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             for (int pass = 0; pass <= nbase; ++pass) {
               ++stale;
               const int cb = (kRtIdxMask - (kb & kRtIdxMask)) / kRtTile;
+              uint32_t hw[kRtTile / 32][WORDS];
+              int ow[kRtTile / 32];
+#pragma unroll
+              for (int i = 0; i < kRtTile / 32; ++i) {
+                const int j = cb * kRtTile + lane + 32 * i;  // below smem_slots: rows past the budget hold zeros
+                ow[i] = j < C ? (int)owner[j] : 0;
+#pragma unroll
+                for (int w = 0; w < WORDS; ++w) hw[i][w] = codes_t[j * WORDS + w];
+              }
               int km = 0;
 #pragma unroll
               for (int i = 0; i < kRtTile / 32; ++i) {
-                const int j = cb * kRtTile + lane + 32 * i;
-                if (j < C && owner[j] < 0) km = max(km, (rt_dist<WORDS>(codes_t + j * WORDS, qr, G) << kRtKeyShift) + (kRtIdxMask - j));
+                int D = 0;
+#pragma unroll
+                for (int g = 0; g < kMaxGroup; ++g) {
+                  if (g < G) {
+#pragma unroll
+                    for (int w = 0; w < WORDS; ++w) D += __popc(hw[i][w] ^ qw[g * WORDS + w]);
+                  }
+                }
+                const int key = (D << kRtKeyShift) + (kRtIdxMask - (cb * kRtTile + lane + 32 * i));
+                km = max(km, ow[i] < 0 ? key : 0);
               }
               km = __reduce_max_sync(0xFFFFFFFFu, km);
               Mx[r * kRtMPitch + cb] = km;  // same value from every lane
