@@ -318,8 +318,8 @@ def run_ours(args, w):
         "roofline_prefill": {"call": "he_prefill_compress (hash K, hash Q, replay, gather)", "bound": "hbm",
                              "achieved": pre_gbs, "peak": peak, "unit": "GB/s", "frac": pre_gbs / peak,
                              "algorithmic_bytes_per_call": pre_bytes,
-                             "note": "the paper-exact sequential replay is integer-ALU/latency bound, not HBM bound"},
-        "gpu_launches": K * R * (5 + T),  # per prefill: hash K, hash Q, schedule, replay, gather; per decode call: 1
+                             "note": "the paper-exact replay is sequential per unit: bound by the step-to-step latency of its resolver warp and by tensor-core tile rate, not by HBM"},
+        "gpu_launches": K * R * (6 + T),  # per prefill: W image, hash K, hash Q, schedule, replay, gather; per decode call: 1
         "input_setup_s": t_gen,
     }
 

@@ -333,21 +333,21 @@ int launch_replay_reg(const ReplayArgs& a, long long units, cudaStream_t stream)
   return launch_replay_smem<WORDS, GT>(a, units, stream);
 }
 
-// Tensor-core replay: one persistent CTA per SM. Used when the whole table of a unit fits its shared-memory layout
-// (budgets up to 4096 slots) and no protected window is set.
-template <int WORDS>
+// Tensor-core replay: one persistent CTA per SM, for budgets up to 12288 slots without a protected window. Up to
+// 4096 slots the unit's tables sit in shared memory, beyond that they are the cache's own arrays.
+template <int WORDS, bool GLOBAL_TABLE>
 int launch_replay_tc(const ReplayArgs& a0, long long units, cudaStream_t stream) {
   ReplayArgs a = a0;
   a.smem_slots = (a.cfg.max_budget + kRtTile - 1) / kRtTile * kRtTile;
-  const size_t smem = rt_layout(WORDS, a.smem_slots, a.cfg.group_size).total;
-  if (int rc = set_smem(prefill_replay_tc_kernel<WORDS>, smem)) return rc;
+  const size_t smem = rt_layout(WORDS, a.smem_slots, a.cfg.group_size, !GLOBAL_TABLE).total;
+  if (int rc = set_smem(prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE>, smem)) return rc;
   int sms = 0;
   if (int rc = sm_count(&sms)) return rc;
   const int nbins = sms < kMaxBins ? sms : kMaxBins;
   prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched);
   HE_CUDA_CHECK(cudaGetLastError());
   const long long grid = units < sms ? units : sms;
-  prefill_replay_tc_kernel<WORDS><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);
+  prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
 }
@@ -363,9 +363,10 @@ int tc_replay_mode() {
 template <int WORDS>
 int launch_replay(const ReplayArgs& a, long long units, cudaStream_t stream) {
   const int mode = tc_replay_mode();
-  if (mode != 0 && a.cfg.max_budget <= kRtMaxSlots && (mode == 2 || a.cfg.max_budget >= 512) && a.cfg.n_sink == 0 &&
+  if (mode != 0 && a.cfg.max_budget <= kRtMaxSlotsGlobal && (mode == 2 || a.cfg.max_budget >= 512) && a.cfg.n_sink == 0 &&
       a.cfg.n_recent == 0)
-    return launch_replay_tc<WORDS>(a, units, stream);
+    return a.cfg.max_budget <= kRtMaxSlots ? launch_replay_tc<WORDS, false>(a, units, stream)
+                                           : launch_replay_tc<WORDS, true>(a, units, stream);
   switch (a.cfg.group_size) {
     case 1: return launch_replay_reg<WORDS, 1>(a, units, stream);
     case 4: return launch_replay_reg<WORDS, 4>(a, units, stream);

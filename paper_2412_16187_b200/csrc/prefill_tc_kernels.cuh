@@ -38,8 +38,8 @@ constexpr int kRtThreads = 416;
 constexpr int kRtMmaWarp = kRtThreads / 32 - 1;
 constexpr int kRtRows = 128;       // steps per block = MMA M
 constexpr int kRtTile = 128;       // slots per tile = MMA N
-constexpr int kRtMaxSlots = 4096;  // 32 tiles: one tile maximum per resolver lane
-constexpr int kRtMPitch = 33;      // words per row of the tile-maximum table (odd: conflict-free column writes)
+constexpr int kRtMaxSlots = 4096;         // largest budget whose code and position tables stay in shared memory
+constexpr int kRtMaxSlotsGlobal = 12288;  // largest budget at all: the tables then live in the cache's own arrays
 constexpr int kRtKeyShift = 14;
 constexpr int kRtIdxMask = (1 << kRtKeyShift) - 1;
 constexpr int kRtStaleLimit = 64;  // repairs after which a block is cut short
@@ -49,16 +49,18 @@ constexpr int kRtAtomBytes = kRtRows * 128;  // one 64-column K-major swizzle at
 struct RtLayout {
   uint32_t a, b, codes, pos, owner, m, rb, dn, qraw, kraw, total;
 };
-__host__ __device__ inline RtLayout rt_layout(int words, int slots, int G) {
+// `slots` is the budget rounded up to whole tiles; the tile-maximum table has an odd pitch (conflict-free column writes).
+__host__ __device__ inline int rt_mpitch(int slots, bool table_in_smem) { return table_in_smem ? kRtMaxSlots / kRtTile + 1 : ((slots / kRtTile) | 1); }
+__host__ __device__ inline RtLayout rt_layout(int words, int slots, int G, bool table_in_smem) {
   RtLayout L;
   const uint32_t atoms = words == 2 ? 2u : 1u;
   uint32_t o = 0;
   L.a = o, o += atoms * kRtAtomBytes;
   L.b = o, o += 2u * atoms * kRtAtomBytes;
-  L.codes = o, o += (uint32_t)slots * words * 4u;
-  L.pos = o, o += (uint32_t)slots * 4u;
+  L.codes = o, o += table_in_smem ? (uint32_t)slots * words * 4u : 0u;
+  L.pos = o, o += table_in_smem ? (uint32_t)slots * 4u : 0u;
   L.owner = o, o += (uint32_t)slots * 2u;
-  L.m = o, o += kRtRows * kRtMPitch * 4u;
+  L.m = o, o += (uint32_t)kRtRows * rt_mpitch(slots, table_in_smem) * 4u;
   L.rb = o, o += kRtRows * 4u;
   L.dn = o, o += kRtRows * kRtRows * 2u;
   L.qraw = o, o += 2u * kRtRows * G * words * 4u;  // two buffers: this block's codes and the next block's
@@ -97,8 +99,10 @@ __device__ __forceinline__ int rt_dist(const uint32_t* h, const uint32_t* q, int
   return D;
 }
 
-template <int WORDS>
-// 13 warps: one scheduler hosts four of them, so 128 registers per thread is the most its 16 K registers allow
+// GLOBAL_TABLE: the unit's code and position tables are the cache's own arrays in global memory (budgets beyond
+// kRtMaxSlots); otherwise they sit in shared memory and are written out when the unit is done.
+// 13 warps: one scheduler hosts four of them, so 128 registers per thread is the most its 16 K registers allow.
+template <int WORDS, bool GLOBAL_TABLE>
 __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const ReplayArgs a) {
   constexpr int ATOMS = WORDS == 2 ? 2 : 1;
   constexpr int KB = 32 * WORDS;             // code columns of the contraction
@@ -119,11 +123,10 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   const long long Cmax = cfg.max_budget;
   const bool write_scores = (cfg.flags & HE_FLAG_WRITE_SCORES) != 0;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(rt_smem_raw) + 1023) & ~(uintptr_t)1023);
-  const RtLayout L = rt_layout(WORDS, a.smem_slots, G);
+  const RtLayout L = rt_layout(WORDS, a.smem_slots, G, !GLOBAL_TABLE);
+  const int mp = GLOBAL_TABLE ? rt_mpitch(a.smem_slots, false) : kRtMaxSlots / kRtTile + 1;  // a constant for the smaller tables
   unsigned char* As = smem + L.a;
   unsigned char* Bs = smem + L.b;
-  uint32_t* codes_t = reinterpret_cast<uint32_t*>(smem + L.codes);
-  int32_t* pos_t = reinterpret_cast<int32_t*>(smem + L.pos);
   int16_t* owner = reinterpret_cast<int16_t*>(smem + L.owner);
   int32_t* Mx = reinterpret_cast<int32_t*>(smem + L.m);
   int32_t* RB = reinterpret_cast<int32_t*>(smem + L.rb);
@@ -183,12 +186,16 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     const uint32_t* qc_u = a.qcodes + unit * a.Nmax * G * WORDS;
     float* sc = a.ca.scores + unit * Cmax;
     const int nbase = (C + kRtTile - 1) / kRtTile;
-    // the first C tokens fill the cache in order
-    for (int j = tid; j < a.smem_slots; j += NT) {
+    uint32_t* codes_t = GLOBAL_TABLE ? a.ca.codes + unit * Cmax * WORDS : reinterpret_cast<uint32_t*>(smem + L.codes);
+    int32_t* pos_t = GLOBAL_TABLE ? a.ca.pos + unit * Cmax : reinterpret_cast<int32_t*>(smem + L.pos);
+    // the first C tokens fill the cache in order; everything beyond `fill` is reset
+    for (int j = tid; j < (GLOBAL_TABLE ? (int)Cmax : a.smem_slots); j += NT) {
 #pragma unroll
       for (int w = 0; w < WORDS; ++w) codes_t[j * WORDS + w] = j < fill0 ? __ldg(kc_u + (long long)j * WORDS + w) : 0u;
       pos_t[j] = j < fill0 ? j : -1;
     }
+    // A table word as the latest step left it (global tables: read past L1, which other warps' stores do not update)
+    auto table_word = [&](int idx) -> uint32_t { return GLOBAL_TABLE ? __ldcg(codes_t + idx) : codes_t[idx]; };
     __syncthreads();
     bool aborted = false;
     const int GW = G * WORDS;
@@ -262,7 +269,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             valid = j < C;
             idx = kRtIdxMask - j;
 #pragma unroll
-            for (int w = 0; w < WORDS; ++w) h[w] = codes_t[j * WORDS + w];
+            for (int w = 0; w < WORDS; ++w) h[w] = valid ? table_word(j * WORDS + w) : 0u;
           } else {  // the block's own keys: plain distances, no index term
             valid = x < rows;
             idx = 0;
@@ -331,7 +338,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(st));
-            Mx[tid * kRtMPitch + i] = __float2int_rn(__uint_as_float(mx));
+            Mx[tid * mp + i] = __float2int_rn(__uint_as_float(mx));
           } else {  // distances of the block's keys: key / 2^14, kept as 16-bit integers
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -354,7 +361,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
         }
         if (ok) {
           int rb = 0;
-          for (int i = 0; i < nbase; ++i) rb = max(rb, Mx[tid * kRtMPitch + i]);
+          for (int i = 0; i < nbase; ++i) rb = max(rb, Mx[tid * mp + i]);
           RB[tid] = rb;
         }
       }
@@ -455,7 +462,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
                 const int j = cb * kRtTile + lane + 32 * i;  // below smem_slots: rows past the budget hold zeros
                 ow[i] = j < C ? (int)owner[j] : 0;
 #pragma unroll
-                for (int w = 0; w < WORDS; ++w) hw[i][w] = codes_t[j * WORDS + w];
+                for (int w = 0; w < WORDS; ++w) hw[i][w] = j < C ? table_word(j * WORDS + w) : 0u;
               }
               int km = 0;
 #pragma unroll
@@ -472,8 +479,11 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
                 km = max(km, ow[i] < 0 ? key : 0);
               }
               km = __reduce_max_sync(0xFFFFFFFFu, km);
-              Mx[r * kRtMPitch + cb] = km;  // same value from every lane
-              kb = __reduce_max_sync(0xFFFFFFFFu, lane < nbase ? Mx[r * kRtMPitch + lane] : 0);
+              Mx[r * mp + cb] = km;  // same value from every lane
+              int rowmax = lane < nbase ? Mx[r * mp + lane] : 0;
+              if (GLOBAL_TABLE)
+                for (int i = lane + 32; i < nbase; i += 32) rowmax = max(rowmax, Mx[r * mp + i]);
+              kb = __reduce_max_sync(0xFFFFFFFFu, rowmax);
               if (kb <= kn || owner[kRtIdxMask - (kb & kRtIdxMask)] < 0) break;
             }
             own_kb = -1;  // exact for this step (or below the best new entry)
@@ -490,7 +500,12 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             }
           } else if (status == 2) {  // Eq. 5 for every slot as the prompt's last step sees the table
             const uint32_t* qr = qb + r * GW;
-            for (int j = lane; j < C; j += 32) sc[j] = -(float)rt_dist<WORDS>(codes_t + j * WORDS, qr, G);
+            for (int j = lane; j < C; j += 32) {
+              uint32_t hj[WORDS];
+#pragma unroll
+              for (int w = 0; w < WORDS; ++w) hj[w] = table_word(j * WORDS + w);
+              sc[j] = -(float)rt_dist<WORDS>(hj, qr, G);
+            }
             scored = true;
           }
         }
@@ -512,9 +527,11 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     const bool scored = write_scores && N > C;
     for (int j = tid; j < Cmax; j += NT) {
       const bool valid = j < fill0;
+      if (!GLOBAL_TABLE) {
 #pragma unroll
-      for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = valid ? codes_t[j * WORDS + w] : 0u;
-      a.ca.pos[unit * Cmax + j] = valid ? pos_t[j] : -1;
+        for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = valid ? codes_t[j * WORDS + w] : 0u;
+        a.ca.pos[unit * Cmax + j] = valid ? pos_t[j] : -1;
+      }
       if (!(valid && scored)) sc[j] = 0.f;
     }
     if (tid == 0) {
