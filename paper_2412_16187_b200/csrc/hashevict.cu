@@ -335,21 +335,29 @@ int launch_replay_reg(const ReplayArgs& a, long long units, cudaStream_t stream)
 
 // Tensor-core replay: one persistent CTA per SM, for budgets up to 12288 slots without a protected window. Up to
 // 4096 slots the unit's tables sit in shared memory, beyond that they are the cache's own arrays.
-template <int WORDS, bool GLOBAL_TABLE>
-int launch_replay_tc(const ReplayArgs& a0, long long units, cudaStream_t stream) {
+template <int WORDS, bool GLOBAL_TABLE, bool FP8>
+int launch_replay_tc_one(const ReplayArgs& a0, long long units, cudaStream_t stream) {
   ReplayArgs a = a0;
   a.smem_slots = (a.cfg.max_budget + kRtTile - 1) / kRtTile * kRtTile;
-  const size_t smem = rt_layout(WORDS, a.smem_slots, a.cfg.group_size, !GLOBAL_TABLE).total;
-  if (int rc = set_smem(prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE>, smem)) return rc;
+  const size_t smem = rt_layout(WORDS, a.smem_slots, a.cfg.group_size, !GLOBAL_TABLE, FP8).total;
+  if (int rc = set_smem(prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8>, smem)) return rc;
   int sms = 0;
   if (int rc = sm_count(&sms)) return rc;
   const int nbins = sms < kMaxBins ? sms : kMaxBins;
   prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched);
   HE_CUDA_CHECK(cudaGetLastError());
   const long long grid = units < sms ? units : sms;
-  prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);
+  prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
+}
+
+// 8-bit operands when the group's code sum fits e5m2 exactly (group sizes up to 7); HE_TC_REPLAY_BF16=1 keeps bf16.
+template <int WORDS, bool GLOBAL_TABLE>
+int launch_replay_tc(const ReplayArgs& a, long long units, cudaStream_t stream) {
+  const char* e = getenv("HE_TC_REPLAY_BF16");
+  if (a.cfg.group_size <= 7 && !(e && e[0] == '1')) return launch_replay_tc_one<WORDS, GLOBAL_TABLE, true>(a, units, stream);
+  return launch_replay_tc_one<WORDS, GLOBAL_TABLE, false>(a, units, stream);
 }
 
 // HE_TC_REPLAY=0 keeps the replay on the CUDA-core kernels, =1 sends every eligible shape to the tensor-core kernel;

@@ -28,6 +28,7 @@
 // barriers as usual, releases tensor memory and returns, and the device error counter is incremented.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "hash_tc_kernels.cuh"
 #include "prefill_kernels.cuh"
@@ -45,18 +46,36 @@ constexpr int kRtIdxMask = (1 << kRtKeyShift) - 1;
 constexpr int kRtStaleLimit = 64;  // repairs after which a block is cut short
 constexpr int kRtAtomBytes = kRtRows * 128;  // one 64-column K-major swizzle atom of a 128-row operand tile
 
+__device__ __forceinline__ void tc_mma_f8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
+
+// e4m3 bit pattern of a small non-negative integer with at most four significant bits (exact).
+__device__ __forceinline__ uint32_t rt_e4m3_of_int(int v) {
+  if (v <= 0) return 0u;
+  const int p = 31 - __clz(v);
+  const uint32_t mant = p >= 3 ? ((uint32_t)v >> (p - 3)) & 7u : ((uint32_t)v << (3 - p)) & 7u;
+  return ((uint32_t)(p + 7) << 3) | mant;
+}
+
 // Byte offsets of the kernel's dynamic shared memory (after rounding its base up to 1024 bytes).
 struct RtLayout {
   uint32_t a, b, codes, pos, owner, m, rb, dn, qraw, kraw, total;
 };
 // `slots` is the budget rounded up to whole tiles; the tile-maximum table has an odd pitch (conflict-free column writes).
 __host__ __device__ inline int rt_mpitch(int slots, bool table_in_smem) { return table_in_smem ? kRtMaxSlots / kRtTile + 1 : ((slots / kRtTile) | 1); }
-__host__ __device__ inline RtLayout rt_layout(int words, int slots, int G, bool table_in_smem) {
+__host__ __device__ inline RtLayout rt_layout(int words, int slots, int G, bool table_in_smem, bool fp8) {
   RtLayout L;
-  const uint32_t atoms = words == 2 ? 2u : 1u;
+  const uint32_t atoms = (words == 2 && !fp8) ? 2u : 1u;  // 8-bit operands: a row of codes and key columns fits 128 bytes
+  const uint32_t stages = fp8 ? 4u : 2u;
   uint32_t o = 0;
   L.a = o, o += atoms * kRtAtomBytes;
-  L.b = o, o += 2u * atoms * kRtAtomBytes;
+  L.b = o, o += stages * atoms * kRtAtomBytes;
   L.codes = o, o += table_in_smem ? (uint32_t)slots * words * 4u : 0u;
   L.pos = o, o += table_in_smem ? (uint32_t)slots * 4u : 0u;
   L.owner = o, o += (uint32_t)slots * 2u;
@@ -102,20 +121,29 @@ __device__ __forceinline__ int rt_dist(const uint32_t* h, const uint32_t* q, int
 // GLOBAL_TABLE: the unit's code and position tables are the cache's own arrays in global memory (budgets beyond
 // kRtMaxSlots); otherwise they sit in shared memory and are written out when the unit is done.
 // 13 warps: one scheduler hosts four of them, so 128 registers per thread is the most its 16 K registers allow.
-template <int WORDS, bool GLOBAL_TABLE>
+// FP8 (group sizes up to 7): operand A in e5m2 (-2^13 u_t with |u_t| <= 7 is exact), operand B in e4m3 (+-1 and
+// the digits of the slot index), K = 32 per instruction: half the operand bytes and three instructions per tile
+// instead of five, four operand stages and four accumulators. The key columns are then
+//   A = [.. | 2^14 | 4096 | 256 | 16 | 1],  B = [.. | G K / 2 | idx >> 12 | (idx >> 8) & 15 | (idx >> 4) & 15 | idx & 15].
+template <int WORDS, bool GLOBAL_TABLE, bool FP8>
 __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const ReplayArgs a) {
-  constexpr int ATOMS = WORDS == 2 ? 2 : 1;
+  constexpr int ATOMS = (WORDS == 2 && !FP8) ? 2 : 1;
   constexpr int KB = 32 * WORDS;             // code columns of the contraction
-  constexpr int KSTEPS = (KB + 16) / 16;     // MMA instructions per tile (the last one holds the three key columns)
-  constexpr int XATOM = KB / 64, XCHUNK = (KB % 64) / 8;  // where the key columns start
+  constexpr int KSTEPS = FP8 ? KB / 32 + 1 : (KB + 16) / 16;  // MMA instructions per tile (the last one holds the key columns)
+  constexpr int ESZ = FP8 ? 1 : 2;           // bytes per operand element
+  constexpr int XATOM = (KB * ESZ) / 128, XCHUNK = ((KB * ESZ) % 128) / 16;  // where the key columns start
+  constexpr int NSTAGE = FP8 ? 4 : 2;        // operand stages = accumulators in tensor memory
   constexpr int NT = kRtThreads;
   extern __shared__ unsigned char rt_smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[8];
+  __shared__ __align__(8) unsigned long long bars[4 * NSTAGE];
   __shared__ uint32_t tmem_base_s;
   __shared__ volatile int abort_flag;
   __shared__ int s_unit, s_done;
   // four code bits -> four bf16 values: operand B takes +-1 (bit set: +1), operand A -+2^13 (bit set: -2^13)
   __shared__ uint2 s_lut_a[16], s_lut_b[16];
+  // 8-bit operands: operand A is summed in f16 (-+2^13 per head) and keeps the high bytes (= e5m2); operand B takes a
+  // whole code byte -> eight e4m3 values of +-1
+  __shared__ uint2 s_lut_b8[FP8 ? 256 : 1];
 
   const he_config& cfg = a.cfg;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -123,7 +151,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   const long long Cmax = cfg.max_budget;
   const bool write_scores = (cfg.flags & HE_FLAG_WRITE_SCORES) != 0;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(rt_smem_raw) + 1023) & ~(uintptr_t)1023);
-  const RtLayout L = rt_layout(WORDS, a.smem_slots, G, !GLOBAL_TABLE);
+  const RtLayout L = rt_layout(WORDS, a.smem_slots, G, !GLOBAL_TABLE, FP8);
   const int mp = GLOBAL_TABLE ? rt_mpitch(a.smem_slots, false) : kRtMaxSlots / kRtTile + 1;  // a constant for the smaller tables
   unsigned char* As = smem + L.a;
   unsigned char* Bs = smem + L.b;
@@ -136,12 +164,12 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
 
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };          // expanders -> MMA: operand stage s is written
-  auto empty_bar = [&](int s) { return bar0 + 8u * (2 + s); };   // MMA -> expanders: stage s has been read
-  auto tfull_bar = [&](int x) { return bar0 + 8u * (4 + x); };   // MMA -> readers: accumulator x is complete
-  auto tempty_bar = [&](int x) { return bar0 + 8u * (6 + x); };  // readers -> MMA: accumulator x is drained
+  auto empty_bar = [&](int s) { return bar0 + 8u * (NSTAGE + s); };       // MMA -> expanders: stage s has been read
+  auto tfull_bar = [&](int x) { return bar0 + 8u * (2 * NSTAGE + x); };   // MMA -> readers: accumulator x is complete
+  auto tempty_bar = [&](int x) { return bar0 + 8u * (3 * NSTAGE + x); };  // readers -> MMA: accumulator x is drained
   if (tid == 0) {
     abort_flag = 0;
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < NSTAGE; ++s) {
       mbar_init(full_bar(s), 128);
       mbar_init(empty_bar(s), 1);
       mbar_init(tfull_bar(s), 1);
@@ -153,11 +181,19 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     auto pick = [&](int bit, uint32_t set, uint32_t clear) { return ((tid >> bit) & 1) ? set : clear; };
     s_lut_b[tid] = make_uint2(pick(0, 0x3F80u, 0xBF80u) | (pick(1, 0x3F80u, 0xBF80u) << 16),
                               pick(2, 0x3F80u, 0xBF80u) | (pick(3, 0x3F80u, 0xBF80u) << 16));
-    s_lut_a[tid] = make_uint2(pick(0, 0xC600u, 0x4600u) | (pick(1, 0xC600u, 0x4600u) << 16),
-                              pick(2, 0xC600u, 0x4600u) | (pick(3, 0xC600u, 0x4600u) << 16));
+    const uint32_t a_set = FP8 ? 0xF000u : 0xC600u, a_clr = FP8 ? 0x7000u : 0x4600u;  // -+2^13 as f16 / bf16
+    s_lut_a[tid] = make_uint2(pick(0, a_set, a_clr) | (pick(1, a_set, a_clr) << 16), pick(2, a_set, a_clr) | (pick(3, a_set, a_clr) << 16));
   }
-  if (warp == kRtMmaWarp) {  // two accumulators of 128 columns
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2 * kRtTile)
+  if (FP8 && tid < 256) {
+    uint32_t lo = 0u, hi = 0u;
+    for (int k = 0; k < 4; ++k) {
+      lo |= (((tid >> k) & 1) ? 0x38u : 0xB8u) << (8 * k);
+      hi |= (((tid >> (k + 4)) & 1) ? 0x38u : 0xB8u) << (8 * k);
+    }
+    s_lut_b8[tid] = make_uint2(lo, hi);
+  }
+  if (warp == kRtMmaWarp) {  // NSTAGE accumulators of 128 columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(NSTAGE * kRtTile)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -165,9 +201,12 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
-  const uint32_t idesc = (1u << 4) /* fp32 accumulate */ | (1u << 7) /* A bf16 */ | (1u << 10) /* B bf16 */ |
-                         ((uint32_t)(kRtTile >> 3) << 17) | ((uint32_t)(kRtRows >> 4) << 24);
+  // instruction descriptor: fp32 accumulate; operand formats bf16 x bf16 (kind::f16: 1, 1) or e5m2 x e4m3
+  // (kind::f8f6f4: 1, 0); both operands K-major; N = 128, M = 128
+  const uint32_t idesc = (1u << 4) | (1u << 7) | ((FP8 ? 0u : 1u) << 10) | ((uint32_t)(kRtTile >> 3) << 17) |
+                         ((uint32_t)(kRtRows >> 4) << 24);
   const uint32_t kconst_bits = __float_as_uint((float)(G * KB / 2) * 16384.f) >> 16;  // exact: G K / 2 <= 256
+  const uint32_t cst_e4m3 = rt_e4m3_of_int(G * KB / 2);
   int it = 0;  // operand tiles processed so far; every role counts the same sequence
 
   for (;;) {
@@ -210,6 +249,40 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     // -+2^13 per bit, exact in packed bf16 adds), then the three key columns 128, 1, G K 2^13.
     auto build_a = [&](int buf, int nrows, int first, int nthreads) {
       const uint32_t* qd = qraw + buf * kRtRows * GW;
+      if (FP8) {  // 16 columns per 16-byte chunk; sums in f16, whose high bytes are the e5m2 values
+        constexpr int NC = KB / 16;
+        for (int item = first; item < kRtRows * (NC + 1); item += nthreads) {
+          const int r = item / (NC + 1), c = item % (NC + 1);
+          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+          if (c < NC) {
+            if (r < nrows) {
+              const int w = c >> 1, sh = (c & 1) * 16;
+              __half2 sm[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) sm[k] = __float2half2_rn(0.f);
+              for (int g = 0; g < G; ++g) {
+                const uint32_t bits = qd[r * GW + g * WORDS + w] >> sh;
+#pragma unroll
+                for (int nb = 0; nb < 4; ++nb) {
+                  const uint2 e = s_lut_a[(bits >> (4 * nb)) & 15u];
+                  sm[2 * nb] = __hadd2(sm[2 * nb], *reinterpret_cast<const __half2*>(&e.x));
+                  sm[2 * nb + 1] = __hadd2(sm[2 * nb + 1], *reinterpret_cast<const __half2*>(&e.y));
+                }
+              }
+              uint32_t wv[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                wv[k] = __byte_perm(*reinterpret_cast<uint32_t*>(&sm[2 * k]), *reinterpret_cast<uint32_t*>(&sm[2 * k + 1]), 0x7531);
+              v = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+            }
+            *reinterpret_cast<uint4*>(As + rt_swz(r, c)) = v;
+          } else {
+            if (r < nrows) v = make_uint4(0x74u | (0x6Cu << 8) | (0x5Cu << 16) | (0x4Cu << 24), 0x3Cu, 0u, 0u);  // 2^14, 4096, 256, 16, 1
+            *reinterpret_cast<uint4*>(As + rt_swz(r, XCHUNK)) = v;
+            *reinterpret_cast<uint4*>(As + rt_swz(r, XCHUNK + 1)) = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+      } else {
       for (int item = first; item < kRtRows * (KB / 8 + 1); item += nthreads) {
         const int r = item / (KB / 8 + 1), c = item % (KB / 8 + 1);
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -235,6 +308,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           *reinterpret_cast<uint4*>(As + XATOM * kRtAtomBytes + rt_swz(r, XCHUNK + 1)) = make_uint4(0u, 0u, 0u, 0u);
         }
       }
+      }
     };
     int t0 = C, cur = 0;
     bool staged = false;  // buffer `cur` and operand A already hold the block that starts at t0
@@ -257,9 +331,9 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
         // two groups of four warps, one per operand stage: group g expands the tiles that go to stage g
         const int x = (tid - 128) & 127, grp = (tid - 128) >> 7;  // x: this thread's row of the tile
         for (int i = 0; i < ntile; ++i) {
-          const int n = it + i, st = n & 1;
-          if (st != grp) continue;
-          if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(st), ((n >> 1) & 1) ^ 1, &abort_flag))) break;
+          const int n = it + i, st = n % NSTAGE, ph = (n / NSTAGE) & 1;
+          if ((n & 1) != grp) continue;
+          if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(st), ph ^ 1, &abort_flag))) break;
           unsigned char* bt = Bs + st * ATOMS * kRtAtomBytes;
           uint32_t h[WORDS];
           bool valid;
@@ -279,7 +353,23 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
           unsigned char* brow = bt + (x >> 3) * 1024 + (x & 7) * 128;  // this row inside each swizzle atom
           const int xs = (x & 7) << 4;
-          if (valid) {
+          if (FP8) {
+            if (valid) {
+#pragma unroll
+              for (int c = 0; c < KB / 16; ++c) {
+                const uint32_t two = h[c >> 1] >> ((c & 1) * 16);
+                const uint2 lo = s_lut_b8[two & 0xFFu], hi = s_lut_b8[(two >> 8) & 0xFFu];
+                *reinterpret_cast<uint4*>(brow + ((c << 4) ^ xs)) = make_uint4(lo.x, lo.y, hi.x, hi.y);
+              }
+              *reinterpret_cast<uint4*>(brow + ((XCHUNK << 4) ^ xs)) =
+                  make_uint4(cst_e4m3 | (rt_e4m3_of_int(idx >> 12) << 8) | (rt_e4m3_of_int((idx >> 8) & 15) << 16) |
+                                 (rt_e4m3_of_int((idx >> 4) & 15) << 24),
+                             rt_e4m3_of_int(idx & 15), 0u, 0u);
+            } else {
+#pragma unroll
+              for (int c = 0; c <= KB / 16; ++c) *reinterpret_cast<uint4*>(brow + ((c << 4) ^ xs)) = zero;
+            }
+          } else if (valid) {
 #pragma unroll
             for (int c = 0; c < KB / 8; ++c) {
               const uint32_t byte = h[c >> 2] >> ((c & 3) * 8);
@@ -301,16 +391,20 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
         if (lane == 0) {
           const uint64_t a_desc0 = umma_desc_k128(smem_u32(As));
           for (int i = 0; i < ntile; ++i) {
-            const int n = it + i, st = n & 1;
-            if (!mbar_wait(tempty_bar(st), ((n >> 1) & 1) ^ 1, &abort_flag)) break;  // readers have drained this accumulator
-            if (!mbar_wait(full_bar(st), (n >> 1) & 1, &abort_flag)) break;
+            const int n = it + i, st = n % NSTAGE, ph = (n / NSTAGE) & 1;
+            if (!mbar_wait(tempty_bar(st), ph ^ 1, &abort_flag)) break;  // readers have drained this accumulator
+            if (!mbar_wait(full_bar(st), ph, &abort_flag)) break;
             tc_fence_after();
             const uint64_t b_desc0 = umma_desc_k128(smem_u32(Bs + st * ATOMS * kRtAtomBytes));
             const uint32_t d_tmem = tmem_base + (uint32_t)(st * kRtTile);
 #pragma unroll
             for (int ks = 0; ks < KSTEPS; ++ks) {
-              const uint32_t off = (uint32_t)(((ks * 16) / 64) * kRtAtomBytes + ((ks * 16) % 64) * 2);
-              tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)(off >> 4), b_desc0 + (uint64_t)(off >> 4), idesc, ks > 0);
+              if (FP8) {  // 32 one-byte columns per instruction
+                tc_mma_f8(d_tmem, a_desc0 + (uint64_t)((ks * 32) >> 4), b_desc0 + (uint64_t)((ks * 32) >> 4), idesc, ks > 0);
+              } else {
+                const uint32_t off = (uint32_t)(((ks * 16) / 64) * kRtAtomBytes + ((ks * 16) % 64) * 2);
+                tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)(off >> 4), b_desc0 + (uint64_t)(off >> 4), idesc, ks > 0);
+              }
             }
             tc_commit(empty_bar(st));   // the operand stage may be rewritten once these MMAs have read it
             tc_commit(tfull_bar(st));   // and the accumulator is complete
@@ -319,8 +413,8 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
       } else {
         bool ok = true;
         for (int i = 0; i < ntile && ok; ++i) {
-          const int n = it + i, st = n & 1;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(st), (n >> 1) & 1, &abort_flag));
+          const int n = it + i, st = n % NSTAGE, ph = (n / NSTAGE) & 1;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(st), ph, &abort_flag));
           if (!ok) break;
           tc_fence_after();
           const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(st * kRtTile);
@@ -545,7 +639,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   __syncthreads();
   if (warp == kRtMmaWarp) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kRtTile) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(NSTAGE * kRtTile) : "memory");
   }
   if (tid == 0 && abort_flag) atomicAdd(&g_tc_error, 1);
 }

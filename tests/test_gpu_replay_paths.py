@@ -1,5 +1,5 @@
-"""The two implementations of the prompt replay (tensor-core kernel, CUDA-core kernels) against the oracle, each
-forced through the environment switch in a fresh process, on shapes that cover one-word and two-word codes, group
+"""The implementations of the prompt replay (tensor-core kernel with 8-bit or bf16 operands, CUDA-core kernels)
+against the oracle, each forced through the environment switches in a fresh process, on shapes that cover one-word and two-word codes, group
 sizes 1, 3 and 4, budgets that are not multiples of the 128-slot tile, ragged budgets, prompts that end inside a
 128-step block, prompts shorter than the budget, and keys with little variety (many equal distances, so the
 lowest-slot rule and the repair of stale tile maxima are exercised)."""
@@ -46,8 +46,9 @@ print("ok")
 """ % (ROOT, os.path.join(ROOT, "tests"))
 
 
-@pytest.mark.parametrize("mode", ["1", "0"], ids=["tensor_cores", "cuda_cores"])
-def test_replay_path(mode):
-    e = dict(os.environ, HE_TC_REPLAY=mode)
+@pytest.mark.parametrize("env", [{"HE_TC_REPLAY": "1"}, {"HE_TC_REPLAY": "1", "HE_TC_REPLAY_BF16": "1"}, {"HE_TC_REPLAY": "0"}],
+                         ids=["tensor_cores_fp8", "tensor_cores_bf16", "cuda_cores"])
+def test_replay_path(env):
+    e = dict(os.environ, **env)
     r = subprocess.run([sys.executable, "-c", SCRIPT], env=e, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and "ok" in r.stdout, r.stdout[-2000:] + r.stderr[-4000:]
