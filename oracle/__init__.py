@@ -49,6 +49,8 @@ def _load():
         lib.orc_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32]
         lib.orc_prefill_codes.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32]
         lib.orc_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32]
+        lib.orc_oneshot_codes.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, i32]
+        lib.orc_oneshot_codes.restype = None
         lib.orc_attend.argtypes = [vp, vp, vp, vp]
         lib.orc_attend.restype = None
         for f in (lib.orc_hash, lib.orc_reset, lib.orc_step_codes, lib.orc_step, lib.orc_prefill_codes, lib.orc_prefill):
@@ -135,6 +137,20 @@ class OracleCache:
         _load().orc_step_codes(ctypes.byref(self._cfg), ctypes.byref(self._ca), _p(qcodes), _p(kcodes), _p(k), _p(v),
                                _p(victim), _p(evicted), self.threads)
         return victim, evicted
+
+    def oneshot_codes(self, kcodes, qcodes, k, v, prompt_len, want_sums=False):
+        """One-shot ranking by averaged Hamming distance (Appendix C) on given codes; fills the cache with the kept tokens."""
+        Nmax = k.shape[2]
+        plen = np.ascontiguousarray(prompt_len, dtype=np.int32)
+        kcodes = np.ascontiguousarray(kcodes, dtype=np.uint32)
+        qcodes = np.ascontiguousarray(qcodes, dtype=np.uint32)
+        assert kcodes.shape == (self.B, self.H, Nmax, self.Wd) and qcodes.shape == (self.B, self.H, Nmax, self.G, self.Wd)
+        assert k.strides == v.strides
+        ks = self._strides(k)
+        sums = np.zeros((self.B, self.H, Nmax), dtype=np.int64) if want_sums else None
+        _load().orc_oneshot_codes(ctypes.byref(self._cfg), ctypes.byref(self._ca), _p(kcodes), _p(qcodes), _p(k), _p(v),
+                                  _p(ks), _p(plen), Nmax, _p(sums), self.threads)
+        return sums
 
     def attend(self, q):
         """Eq. 1 over the compressed cache (Algorithm 1 line 6). q [B, H*G, d] -> fp64 [B, H*G, d]."""

@@ -31,6 +31,7 @@
 // invariants; codes == hash(K) for every slot; prefill == reset + N steps; the storage closed
 // form of Section 4.7; orc_attend against a library softmax-attention in fp64, a single-slot cache, equal keys (mean
 // of V), invariance to the slot order. Parity unpinned: none.
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -283,6 +284,68 @@ extern "C" void orc_prefill(const orc_config* cfg, orc_cache* ca, const float* W
   orc_prefill_codes(cfg, ca, kc.data(), qc.data(), k, v, kv_strides, prompt_len, max_prompt_len, threads);
 }
 
+
+// One-shot ranking by averaged Hamming distance (Appendix C: "the average Hamming distance between the key code of
+// token i and the query codes of all tokens j > i", tokens sorted from lowest to highest average). This is the
+// paper's global-ranking simulation, NOT the procedure of Section 3; here it is written out as a prompt-compression
+// variant: the C best-ranked tokens stay. Per unit, with the group's G query heads summed as in Eq. 5:
+//   S_i = sum_{j > i} sum_g popc(h(k_i) xor h(q_{j,g})),   n_i = N - 1 - i,   average_i = S_i / n_i  (0 when n_i = 0).
+// Order: tokens inside the protected windows (i < n_sink or i >= N - n_recent) first, in token order; then by
+// average, compared exactly as fractions (S_a n_b < S_b n_a); equal averages by token index. The first min(N, C)
+// tokens of that order are kept and stored in token order: slot s holds the s-th kept token (its K, V, code and
+// position; score = -(float)S / (float)n, 0 when n = 0). kcodes [B, Hkv, Nmax, Wd]; qcodes [B, Hkv, Nmax, G, Wd];
+// sums_out [B, Hkv, Nmax] int64 (nullable) receives S_i. The cache is reset first.
+extern "C" void orc_oneshot_codes(const orc_config* cfg, orc_cache* ca, const uint32_t* kcodes, const uint32_t* qcodes,
+                                  const void* k, const void* v, const int64_t* kv_strides, const int32_t* prompt_len,
+                                  int32_t max_prompt_len, int64_t* sums_out, int32_t threads) {
+  const int Wd = words_of(cfg->hash_bits), G = cfg->group_size, d = cfg->head_dim, es = esize(cfg->dtype);
+  const int64_t units = (int64_t)cfg->batch * cfg->n_kv_heads, Nmax = max_prompt_len, Cmax = cfg->max_budget;
+  orc_reset(cfg, ca);
+  for_units(units, threads, [=](int64_t u) {
+    const int64_t s = u / cfg->n_kv_heads, h = u % cfg->n_kv_heads;
+    const int32_t C = ca->budget[s], N = prompt_len[s];
+    std::vector<int64_t> S(N, 0);
+    for (int32_t i = 0; i < N; ++i) {
+      const uint32_t* hi = kcodes + (u * Nmax + i) * Wd;
+      int64_t acc = 0;
+      for (int32_t j = i + 1; j < N; ++j)
+        for (int g = 0; g < G; ++g) {
+          const uint32_t* hq = qcodes + ((u * Nmax + j) * G + g) * Wd;
+          for (int w = 0; w < Wd; ++w) acc += __builtin_popcount(hi[w] ^ hq[w]);
+        }
+      S[i] = acc;
+      if (sums_out) sums_out[u * Nmax + i] = acc;
+    }
+    std::vector<int32_t> order(N);
+    for (int32_t i = 0; i < N; ++i) order[i] = i;
+    auto prot = [&](int32_t i) { return i < cfg->n_sink || i >= N - cfg->n_recent; };
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+      const bool pa = prot(a), pb = prot(b);
+      if (pa != pb) return pa;
+      if (pa) return a < b;
+      const int64_t na = N - 1 - a > 0 ? N - 1 - a : 1, nb = N - 1 - b > 0 ? N - 1 - b : 1;  // S = 0 when n = 0
+      const int64_t lhs = S[a] * nb, rhs = S[b] * na;
+      if (lhs != rhs) return lhs < rhs;
+      return a < b;
+    });
+    const int32_t keep = N < C ? N : C;
+    std::vector<int32_t> kept(order.begin(), order.begin() + keep);
+    std::sort(kept.begin(), kept.end());
+    for (int32_t sl = 0; sl < keep; ++sl) {
+      const int32_t t = kept[sl];
+      const int64_t slot = u * Cmax + sl;
+      const int64_t off = (s * kv_strides[0] + h * kv_strides[1] + (int64_t)t * kv_strides[2]) * es;
+      std::memcpy((char*)ca->k_cache + slot * d * es, (const char*)k + off, (size_t)d * es);
+      std::memcpy((char*)ca->v_cache + slot * d * es, (const char*)v + off, (size_t)d * es);
+      for (int w = 0; w < Wd; ++w) ca->codes[slot * Wd + w] = kcodes[(u * Nmax + t) * Wd + w];
+      ca->pos[slot] = t;
+      const int64_t n = N - 1 - t;
+      ca->scores[slot] = n > 0 ? -((float)S[t] / (float)n) : 0.0f;
+    }
+    ca->fill[u] = keep;
+    ca->next_pos[u] = N;
+  });
+}
 
 // Eq. 1 over the compressed cache (Algorithm 1 line 6): for every unit and each of its G query heads,
 //   out[g] = sum_j softmax_j( q_g . K_j / sqrt(d) ) V_j   over the valid slots j < fill.

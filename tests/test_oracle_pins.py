@@ -317,3 +317,75 @@ def test_attend_special_cases():
     oc.k_cache[0, 0, :5] = oc.k_cache[0, 0, perm]
     oc.v_cache[0, 0, :5] = oc.v_cache[0, 0, perm]
     np.testing.assert_allclose(oc.attend(q), a, rtol=1e-12, atol=1e-13)  # the slot order does not matter
+
+
+# ---------------------------------------------------------------- one-shot averaged-Hamming ranking (Appendix C)
+
+def test_oneshot_worked_example():
+    # b = 2, G = 1, three tokens, budget 2. Key codes 00, 11, 01; query codes (of tokens 1, 2) 01, 10.
+    # S_0 = |00^01| + |00^10| = 2 over n = 2 -> 1; S_1 = |11^10| = 1 over n = 1 -> 1; token 2 has no later query -> 0.
+    # Order: token 2, then the tie at 1 by index: 0, 1. Kept: {0, 2}, stored in token order.
+    oc = oracle.OracleCache(1, 1, 1, 8, 2, 4, [2], "f32")
+    kc = np.array([0b00, 0b11, 0b01], dtype=np.uint32).reshape(1, 1, 3, 1)
+    qc = np.array([0b11, 0b01, 0b10], dtype=np.uint32).reshape(1, 1, 3, 1, 1)  # token 0's query is never used
+    k = np.arange(24, dtype=np.float32).reshape(1, 1, 3, 8)
+    v = -k
+    sums = oc.oneshot_codes(kc, qc, k, v, [3], want_sums=True)
+    assert sums[0, 0].tolist() == [2, 1, 0]
+    assert oc.pos[0, 0].tolist() == [0, 2, -1, -1] and oc.fill[0, 0] == 2 and oc.next_pos[0, 0] == 3
+    assert oc.scores[0, 0].tolist() == [-1.0, 0.0, 0.0, 0.0]
+    assert np.array_equal(oc.k_cache[0, 0, 1], k[0, 0, 2]) and np.array_equal(oc.v_cache[0, 0, 0], v[0, 0, 0])
+    assert oc.codes[0, 0, :2, 0].tolist() == [0b00, 0b01]
+
+
+@pytest.mark.parametrize("G,b,n_sink,n_recent", [(1, 8, 0, 0), (4, 40, 0, 0), (2, 64, 3, 5), (3, 16, 0, 2)])
+def test_oneshot_against_per_bit_counts_and_exact_fractions(G, b, n_sink, n_recent):
+    from fractions import Fraction
+
+    rng = np.random.default_rng(11 + G)
+    B, H, N, C, d = 2, 2, 57, 20, 8
+    Wd = oracle.words(b)
+    mask = [(1 << min(32, b - 32 * w)) - 1 for w in range(Wd)]
+    kc = rng.integers(0, 2**32, size=(B, H, N, Wd), dtype=np.uint64).astype(np.uint32) & np.array(mask, dtype=np.uint32)
+    qc = rng.integers(0, 2**32, size=(B, H, N, G, Wd), dtype=np.uint64).astype(np.uint32) & np.array(mask, dtype=np.uint32)
+    kc[0, 0, 5:9] = kc[0, 0, 4]  # equal keys next to each other: equal sums only if their later queries agree
+    qc[1, 1, 30:] = qc[1, 1, 29]  # a constant tail of queries: many equal averages
+    plen = np.array([N, 13], dtype=np.int32)  # the second sequence is shorter than its budget
+    oc = oracle.OracleCache(B, H, G, d, b, C, [C, C - 3], "f32", n_sink=n_sink, n_recent=n_recent)
+    k = rng.standard_normal((B, H, N, d)).astype(np.float32)
+    v = rng.standard_normal((B, H, N, d)).astype(np.float32)
+    sums = oc.oneshot_codes(kc, qc, k, v, plen, want_sums=True)
+    for s in range(B):
+        n_tok, cap = int(plen[s]), int(oc.budget[s])
+        for h in range(H):
+            kb = unpack(kc[s, h, :n_tok], b).astype(np.int64)          # [N, b]
+            qb = unpack(qc[s, h, :n_tok].reshape(n_tok * G, Wd), b).reshape(n_tok, G, b).astype(np.int64).sum(1)  # ones per bit
+            later = np.concatenate([np.cumsum(qb[::-1], axis=0)[::-1][1:], np.zeros((1, b), dtype=np.int64)])  # tokens j > i
+            m = (n_tok - 1 - np.arange(n_tok))[:, None] * G
+            want = np.where(kb == 1, m - later, later).sum(1)  # a set key bit differs from the zeros, a clear one from the ones
+            assert np.array_equal(sums[s, h, :n_tok], want)
+            prot = [i for i in range(n_tok) if i < n_sink or i >= n_tok - n_recent]
+            rest = sorted((i for i in range(n_tok) if i not in prot),
+                          key=lambda i: (Fraction(int(want[i]), max(1, n_tok - 1 - i)), i))
+            keep = sorted((prot + rest)[:min(n_tok, cap)])
+            fill = int(oc.fill[s, h])
+            assert fill == len(keep) and oc.pos[s, h, :fill].tolist() == keep and np.all(oc.pos[s, h, fill:] == -1)
+            assert oc.next_pos[s, h] == n_tok
+            for sl, t in enumerate(keep):
+                assert np.array_equal(oc.codes[s, h, sl], kc[s, h, t]) and np.array_equal(oc.k_cache[s, h, sl], k[s, h, t])
+                n = n_tok - 1 - t
+                assert oc.scores[s, h, sl] == (-(np.float32(want[t]) / np.float32(n)) if n > 0 else 0.0)
+
+
+def test_oneshot_special_cases():
+    b, G, N, C = 16, 2, 12, 5
+    oc = oracle.OracleCache(1, 1, G, 8, b, C, [C], "f32")
+    k = np.zeros((1, 1, N, 8), dtype=np.float32)
+    kc = np.full((1, 1, N, 1), 0x1234, dtype=np.uint32)
+    same = np.full((1, 1, N, G, 1), 0x1234, dtype=np.uint32)
+    sums = oc.oneshot_codes(kc, same, k, k, [N], want_sums=True)
+    assert not sums.any() and oc.pos[0, 0].tolist() == [0, 1, 2, 3, 4]  # all averages equal: the lowest indices stay
+    sums = oc.oneshot_codes(kc, same ^ np.uint32(0xFFFF), k, k, [N], want_sums=True)
+    assert sums[0, 0].tolist() == [G * b * (N - 1 - i) for i in range(N)]  # complementary codes: every bit differs
+    # average G*b for all but the last token (0): the last token first, then the lowest indices
+    assert oc.pos[0, 0].tolist() == [0, 1, 2, 3, N - 1]
