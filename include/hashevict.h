@@ -163,6 +163,25 @@ int he_prefill_compress_host(const he_config* cfg, const he_cache* cache, const 
                              int32_t* fill_host, void* staging, size_t staging_bytes, void* stream);
 
 /*
+ * he_prefill_oneshot - prompt compression by the one-shot ranking of Appendix C instead of Algorithm 1: for every
+ * prompt token i the Hamming distance of its key code to the query codes of all later tokens j > i (summed over the
+ * group's G query heads as in Eq. 5) is averaged over those tokens, and the min(N, C) tokens with the lowest average
+ * stay. The paper uses this ranking only to analyse the method; it is NOT the procedure of Section 3 and gives a
+ * different cache. Order: tokens inside the protected windows (i < n_sink or i >= N - n_recent) first, in token
+ * order; then by average, compared exactly as fractions; equal averages by token index; the prompt's last token has
+ * no later query and counts as average 0. Kept tokens are stored in token order: slot s holds the s-th kept token
+ * (K, V, code, position; score = -(float)S / (float)n with S the summed distance and n = N - 1 - i, 0 when n = 0);
+ * fill = min(N, C), next_pos = N, everything beyond fill is reset. Arguments, layouts, strides and errors are those
+ * of he_prefill_compress, except: workspace >= he_oneshot_workspace_bytes(cfg, max_prompt_len) bytes;
+ * max_prompt_len <= 32768; sums_out (device, nullable) [B, Hkv, max_prompt_len] int64 receives S for every prompt
+ * token (entries beyond a sequence's length are not written). All arithmetic is integer except the stored score.
+ */
+size_t he_oneshot_workspace_bytes(const he_config* cfg, int32_t max_prompt_len);
+int he_prefill_oneshot(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
+                       const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len,
+                       int32_t max_prompt_len, void* workspace, size_t workspace_bytes, long long* sums_out, void* stream);
+
+/*
  * he_prefill_compress_noalloc - he_prefill_compress for callers that cannot obtain device memory for the
  * prompt-code workspace. (The paper has no counterpart: this is a packaging variant, the computation and the
  * results are those of he_prefill_compress.)

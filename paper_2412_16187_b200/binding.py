@@ -36,7 +36,7 @@ class he_cache(ctypes.Structure):
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
     "he_decode_staging_bytes", "he_decode_step_host", "he_prefill_staging_bytes", "he_prefill_compress_host",
-    "he_prefill_compress_noalloc", "he_attend", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
+    "he_prefill_compress_noalloc", "he_attend", "he_prefill_oneshot", "he_oneshot_workspace_bytes", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
 )
 
 _lib = None
@@ -67,6 +67,9 @@ def lib():
     L.he_prefill_staging_bytes.restype = sz
     L.he_prefill_compress_host.argtypes = [cfgp, cap, vp, vp, vp, vp, i32, vp, vp, sz, vp]
     L.he_prefill_compress_noalloc.argtypes = [cfgp, cap, vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), vp, i32, vp]
+    L.he_prefill_oneshot.argtypes = [cfgp, cap, vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), vp, i32, vp, sz, vp, vp]
+    L.he_oneshot_workspace_bytes.argtypes = [cfgp, i32]
+    L.he_oneshot_workspace_bytes.restype = sz
     L.he_attend.argtypes = [cfgp, cap, vp, vp, vp]
     L.he_attend.restype = ctypes.c_int
     L.he_step_scratch_bytes.argtypes = [cfgp]
@@ -197,6 +200,19 @@ class HashEvictCache:
         _check(lib().he_prefill_compress(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q), _ptr(k), _ptr(v),
                                          i64x3(*q.stride()[:3]), i64x3(*k.stride()[:3]), _ptr(prompt_len), nmax,
                                          _ptr(ws), ws.numel(), _stream(stream)))
+
+    def prefill_oneshot(self, q, k, v, prompt_len, max_prompt_len=None, sums_out=None, stream=None):
+        """he_prefill_oneshot: the averaged-Hamming ranking of Appendix C instead of Algorithm 1 (same arguments as
+        prefill_compress; sums_out int64 [B, H, Nmax] optionally receives the summed distances)."""
+        nmax = k.shape[2] if max_prompt_len is None else max_prompt_len
+        need = lib().he_oneshot_workspace_bytes(ctypes.byref(self.cfg), nmax)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.k_cache.device)
+        assert q.stride(3) == 1 and k.stride(3) == 1 and k.stride() == v.stride()
+        i64x3 = ctypes.c_int64 * 3
+        _check(lib().he_prefill_oneshot(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q), _ptr(k), _ptr(v),
+                                        i64x3(*q.stride()[:3]), i64x3(*k.stride()[:3]), _ptr(prompt_len), nmax,
+                                        _ptr(self._ws), self._ws.numel(), _ptr(sums_out), _stream(stream)))
 
     def prefill_compress_noalloc(self, q, k, v, prompt_len, max_prompt_len=None, stream=None):
         """he_prefill_compress_noalloc: same call, prompt codes go to the library's built-in scratch (no workspace,

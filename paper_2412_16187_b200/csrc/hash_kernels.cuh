@@ -22,6 +22,7 @@ struct HashJob {
   long long Nmax;
   const int32_t* prompt_len;
   const int32_t* budget;
+  int q_all;            // mode 2: hash the queries of every prompt token, not only of those that evict
   const void* w_image;  // optional: the tensor-core kernel's shared-memory image of W's three bf16 terms (build_w_image_kernel)
 };
 
@@ -56,7 +57,7 @@ __global__ void __launch_bounds__(kHashThreads) hash_rows_kernel(const HashJob j
       out_base = ((long long)s * job.Hkv + hh) * job.Nmax * WORDS;
       out_stride = WORDS;
     } else {
-      r_begin = C < N ? C : N;  // queries of appended tokens are never read
+      r_begin = job.q_all ? 0 : (C < N ? C : N);  // queries of appended tokens are never read by Algorithm 1
       const long long unit = (long long)s * job.Hkv + hh / job.G;
       out_base = (unit * job.Nmax * job.G + hh % job.G) * WORDS;
       out_stride = (long long)job.G * WORDS;

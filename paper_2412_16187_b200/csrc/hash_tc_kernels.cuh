@@ -182,7 +182,7 @@ __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long lo
       o->out_base = ((long long)s * job.Hkv + hh) * job.Nmax * WORDS;
       o->out_stride = WORDS;
     } else {
-      r_begin = C < N ? C : N;
+      r_begin = job.q_all ? 0 : (C < N ? C : N);
       const long long unit = (long long)s * job.Hkv + hh / job.G;
       o->out_base = (unit * job.Nmax * job.G + hh % job.G) * WORDS;
       o->out_stride = (long long)job.G * WORDS;

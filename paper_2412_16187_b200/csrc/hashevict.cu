@@ -24,6 +24,7 @@
 #include "hash_kernels.cuh"
 #include "hash_tc_kernels.cuh"
 #include "hashevict.h"
+#include "oneshot_kernels.cuh"
 #include "prefill_kernels.cuh"
 #include "prefill_tc_kernels.cuh"
 
@@ -498,9 +499,23 @@ size_t he_workspace_bytes(const he_config* cfg, int32_t max_prompt_len) {
   return kbytes + qbytes + align_up(sched_words((long long)units) * 4, 256) + align_up(kWImageBytes, 256) + 256;
 }
 
-int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
-                        const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len,
-                        int32_t max_prompt_len, void* workspace, size_t workspace_bytes, void* stream) {
+size_t he_oneshot_workspace_bytes(const he_config* cfg, int32_t max_prompt_len) {
+  const size_t base = he_workspace_bytes(cfg, max_prompt_len);
+  if (base == 0) return 0;
+  const size_t tokens = (size_t)cfg->batch * cfg->n_kv_heads * (size_t)max_prompt_len;
+  return base + align_up(tokens * 4, 256) + align_up(tokens * 8, 256);
+}
+
+}  // extern "C"
+
+namespace {
+
+// Shared body of he_prefill_compress (oneshot = false: Algorithm 1 replayed over the prompt) and he_prefill_oneshot
+// (oneshot = true: the averaged-Hamming ranking of Appendix C): validation, Eq. 2 on the prompt's keys and queries,
+// the selection kernel(s), the gather of the surviving K / V rows.
+int prefill_impl(bool oneshot, const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
+                 const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len, int32_t max_prompt_len,
+                 void* workspace, size_t workspace_bytes, long long* sums_out, void* stream) {
   if (int rc = check_config(cfg, true)) return rc;
   if (int rc = check_cache(cache)) return rc;
   if (!q || !k || !v || !q_strides || !kv_strides || !prompt_len || !workspace)
@@ -512,8 +527,9 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
       return fail(HE_ERR_INVALID_ARG, "strides must keep every row 16-byte aligned");
   if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return fail(HE_ERR_INVALID_ARG, "q, k, v must be 16-byte aligned");
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return fail(HE_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
-  const size_t need = he_workspace_bytes(cfg, max_prompt_len);
+  const size_t need = oneshot ? he_oneshot_workspace_bytes(cfg, max_prompt_len) : he_workspace_bytes(cfg, max_prompt_len);
   if (workspace_bytes < need) return fail(HE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+  if (oneshot && max_prompt_len > 32768) return fail(HE_ERR_UNSUPPORTED, "one-shot ranking: max_prompt_len %d > 32768", max_prompt_len);
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const long long units = (long long)cfg->batch * cfg->n_kv_heads;
@@ -547,6 +563,7 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
   job.x = q;
   job.out = qcodes;
   job.mode = 2;
+  job.q_all = oneshot ? 1 : 0;  // the ranking reads the queries of all later tokens, Algorithm 1 only those that evict
   job.heads = cfg->n_kv_heads * G;
   job.s0 = q_strides[0];
   job.s1 = q_strides[1];
@@ -556,8 +573,18 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
   // phase 2: the sequential replay of Algorithm 1 over the prompt, one CTA per unit
   int32_t* sched = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(qcodes) +
                                               align_up((size_t)units * max_prompt_len * G * Wd * 4, 256));
-  ReplayArgs ra{*cfg, *cache, kcodes, qcodes, prompt_len, max_prompt_len, cfg->max_budget, sched};
-  if (int rc = (Wd == 1 ? launch_replay<1>(ra, units, st) : launch_replay<2>(ra, units, st))) return rc;
+  if (oneshot) {
+    if (units > 0x7FFFFFFF) return fail(HE_ERR_UNSUPPORTED, "too many units");
+    char* extra = static_cast<char*>(workspace) + he_workspace_bytes(cfg, max_prompt_len);
+    OneshotArgs oa{*cfg, *cache, kcodes, qcodes, prompt_len, max_prompt_len, reinterpret_cast<int32_t*>(extra),
+                   reinterpret_cast<unsigned long long*>(extra + align_up((size_t)units * max_prompt_len * 4, 256)), sums_out};
+    if (Wd == 1) oneshot_rank_kernel<1><<<(unsigned)units, kOneshotThreads, 0, st>>>(oa);
+    else oneshot_rank_kernel<2><<<(unsigned)units, kOneshotThreads, 0, st>>>(oa);
+    HE_CUDA_CHECK(cudaGetLastError());
+  } else {
+    ReplayArgs ra{*cfg, *cache, kcodes, qcodes, prompt_len, max_prompt_len, cfg->max_budget, sched};
+    if (int rc = (Wd == 1 ? launch_replay<1>(ra, units, st) : launch_replay<2>(ra, units, st))) return rc;
+  }
 
   // phase 3: surviving K / V rows into their slots
   GatherArgs ga{*cfg, *cache, k, v, kv_strides[0], kv_strides[1], kv_strides[2]};
@@ -567,6 +594,24 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
   prefill_gather_kernel<<<dim3((unsigned)gx, (unsigned)units), kGatherThreads, 0, st>>>(ga);
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
+                        const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len,
+                        int32_t max_prompt_len, void* workspace, size_t workspace_bytes, void* stream) {
+  return prefill_impl(false, cfg, cache, q, k, v, q_strides, kv_strides, prompt_len, max_prompt_len, workspace, workspace_bytes,
+                      nullptr, stream);
+}
+
+int he_prefill_oneshot(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
+                       const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len,
+                       int32_t max_prompt_len, void* workspace, size_t workspace_bytes, long long* sums_out, void* stream) {
+  return prefill_impl(true, cfg, cache, q, k, v, q_strides, kv_strides, prompt_len, max_prompt_len, workspace, workspace_bytes,
+                      sums_out, stream);
 }
 
 int he_prefill_compress_noalloc(const he_config* cfg, const he_cache* cache, const void* q, const void* k,

@@ -1,0 +1,177 @@
+// he_prefill_oneshot: prompt compression by the averaged-Hamming ranking of Appendix C (the paper's global-ranking
+// simulation; NOT the procedure of Section 3). Per unit and prompt token i, with the group's G query heads summed as
+// in Eq. 5:
+//   S_i = sum_{j > i} sum_g popc(h(k_i) xor h(q_{j,g})),   average_i = S_i / (N - 1 - i)   (0 for the last token);
+// the min(N, C) tokens with the lowest average stay (protected windows first, equal averages by token index).
+//
+// The double sum is linear in per-bit counts, so no N x N pass is needed: with later_i[k] = number of (j > i, g) whose
+// query code has bit k set,  S_i = sum_k ( bit_k(h(k_i)) ? (N-1-i) G - later_i[k] : later_i[k] ).  A lane owns bit k
+// (and k + 32), keeps later[k] in a register while its warp walks a chunk of tokens backwards, and one redux.sync
+// per token adds the lanes' terms. O(N (G + b)) integer work per unit, all of it exact.
+//
+// Selection is exact as well: averages are compared through the key floor(S 2^32 / n), which orders any two
+// fractions with denominators below 2^15 like the fractions themselves (they differ by at least 2^-30), the token
+// index is appended, and a radix select (8 bits per pass) finds the min(N, C)-th smallest key.
+#pragma once
+#include "common.cuh"
+
+namespace he {
+
+struct OneshotArgs {
+  he_config cfg;
+  he_cache ca;
+  const uint32_t* kcodes;  // [units, Nmax, Wd]
+  const uint32_t* qcodes;  // [units, Nmax, G, Wd]
+  const int32_t* prompt_len;
+  long long Nmax;
+  int32_t* sums;             // scratch [units, Nmax]: S_i
+  unsigned long long* keys;  // scratch [units, Nmax]: selection keys
+  long long* sums_out;       // optional [units, Nmax]: S_i for the caller
+};
+
+constexpr int kOneshotThreads = 256;
+constexpr int kOneshotWarps = kOneshotThreads / 32;
+constexpr unsigned long long kOneshotRanked = 1ull << 57;  // set in the keys of tokens outside the protected windows
+
+template <int WORDS>
+__global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const OneshotArgs a) {
+  __shared__ int chunk_cnt[kOneshotWarps][32 * WORDS];
+  __shared__ unsigned int hist[256];
+  __shared__ unsigned long long s_prefix;
+  __shared__ int s_want;
+  __shared__ int s_scan[kOneshotThreads];
+  const he_config& cfg = a.cfg;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long unit = blockIdx.x;
+  const int s = (int)(unit / cfg.n_kv_heads);
+  const int G = cfg.group_size, GW = G * WORDS;
+  const long long Cmax = cfg.max_budget;
+  const int C = min(a.ca.budget[s], (int)Cmax);
+  const int N = a.prompt_len[s];
+  const int keep = N < C ? N : C;
+  const uint32_t* kc_u = a.kcodes + unit * a.Nmax * WORDS;
+  const uint32_t* qc_u = a.qcodes + unit * a.Nmax * GW;
+  int32_t* S = a.sums + unit * a.Nmax;
+  unsigned long long* keys = a.keys + unit * a.Nmax;
+
+  // ---- (1) S_i. Tokens are split into one contiguous chunk per warp; a lane counts the ones of its bits.
+  const int chunk = (N + kOneshotWarps - 1) / kOneshotWarps;
+  const int lo = min(N, warp * chunk), hi = min(N, lo + chunk);
+  int cnt[WORDS];
+#pragma unroll
+  for (int w = 0; w < WORDS; ++w) cnt[w] = 0;
+  for (int j = lo; j < hi; ++j) {  // ones per bit over this warp's chunk
+    for (int g = 0; g < G; ++g) {
+#pragma unroll
+      for (int w = 0; w < WORDS; ++w) cnt[w] += (__ldg(qc_u + (long long)j * GW + g * WORDS + w) >> lane) & 1u;
+    }
+  }
+#pragma unroll
+  for (int w = 0; w < WORDS; ++w) chunk_cnt[warp][w * 32 + lane] = cnt[w];
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < WORDS; ++w) {  // ones per bit over all later chunks
+    cnt[w] = 0;
+    for (int x = warp + 1; x < kOneshotWarps; ++x) cnt[w] += chunk_cnt[x][w * 32 + lane];
+  }
+  for (int i = hi - 1; i >= lo; --i) {  // cnt = ones per bit over the tokens j > i
+    const int m = (N - 1 - i) * G;
+    int term = 0;
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w) {
+      const uint32_t hbit = (__ldg(kc_u + (long long)i * WORDS + w) >> lane) & 1u;
+      term += hbit ? m - cnt[w] : cnt[w];
+    }
+    const int Si = __reduce_add_sync(0xFFFFFFFFu, term);
+    if (lane == 0) {
+      S[i] = Si;
+      if (a.sums_out != nullptr) a.sums_out[unit * a.Nmax + i] = Si;
+    }
+    for (int g = 0; g < G; ++g) {
+#pragma unroll
+      for (int w = 0; w < WORDS; ++w) cnt[w] += (__ldg(qc_u + (long long)i * GW + g * WORDS + w) >> lane) & 1u;
+    }
+  }
+  __syncthreads();
+
+  // ---- (2) keys: protected tokens sort first in token order, the others by average, then index
+  for (int i = tid; i < N; i += kOneshotThreads) {
+    const bool prot = i < cfg.n_sink || i >= N - cfg.n_recent;
+    const int n = N - 1 - i;
+    unsigned long long key = (unsigned long long)i;
+    if (!prot) {
+      const unsigned long long q = n > 0 ? ((unsigned long long)(uint32_t)S[i] << 32) / (unsigned long long)n : 0ull;
+      key = kOneshotRanked | (q << 15) | (unsigned long long)i;
+    }
+    keys[i] = key;
+  }
+  __syncthreads();
+
+  // ---- (3) the keep-th smallest key by radix select, 8 bits per pass from the top (keys are distinct)
+  unsigned long long thresh = ~0ull;
+  if (keep < N) {
+    if (tid == 0) {
+      s_prefix = 0ull;
+      s_want = keep;
+    }
+    for (int shift = 56; shift >= 0; shift -= 8) {
+      hist[tid] = 0u;  // 256 threads, 256 bins
+      __syncthreads();
+      const unsigned long long prefix = s_prefix;
+      for (int i = tid; i < N; i += kOneshotThreads) {
+        const unsigned long long key = keys[i];
+        if (shift == 56 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int want = s_want, bin = 0;
+        while (bin < 255 && (int)hist[bin] < want) want -= (int)hist[bin++];
+        s_want = want;
+        s_prefix = (prefix << 8) | (unsigned long long)bin;
+      }
+      __syncthreads();
+    }
+    thresh = s_prefix;
+  }
+
+  // ---- (4) kept tokens in token order: slot = number of kept tokens before this one
+  const int per = (N + kOneshotThreads - 1) / kOneshotThreads;
+  const int b0 = min(N, tid * per), b1 = min(N, b0 + per);
+  int mine = 0;
+  for (int i = b0; i < b1; ++i) mine += keys[i] <= thresh ? 1 : 0;
+  s_scan[tid] = mine;
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+    for (int t = 0; t < kOneshotThreads; ++t) {
+      const int c = s_scan[t];
+      s_scan[t] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
+  int slot = s_scan[tid];
+  for (int i = b0; i < b1; ++i) {
+    if (keys[i] <= thresh) {
+      const long long dst = unit * Cmax + slot;
+#pragma unroll
+      for (int w = 0; w < WORDS; ++w) a.ca.codes[dst * WORDS + w] = kc_u[(long long)i * WORDS + w];
+      a.ca.pos[dst] = i;
+      const int n = N - 1 - i;
+      a.ca.scores[dst] = n > 0 ? -((float)S[i] / (float)n) : 0.f;
+      ++slot;
+    }
+  }
+  for (int j = keep + tid; j < Cmax; j += kOneshotThreads) {  // everything beyond `fill` is reset
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = 0u;
+    a.ca.pos[unit * Cmax + j] = -1;
+    a.ca.scores[unit * Cmax + j] = 0.f;
+  }
+  if (tid == 0) {
+    a.ca.fill[unit] = keep;
+    a.ca.next_pos[unit] = N;
+  }
+}
+
+}  // namespace he
