@@ -213,7 +213,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = job.d, b = job.b;
   const int KH = d / 64;  // 64-channel halves (128 bytes of bf16 each)
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
+  // rounded up to 1024 bytes by an offset from the array itself: the accesses stay shared-memory accesses
+  unsigned char* smem = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
   unsigned char* Bs = smem;
   const int b_tile_bytes = N * 128;
   unsigned char* As = Bs + 3 * KH * b_tile_bytes;  // N * 128 is a multiple of 1024 for N = 32, 64

@@ -150,7 +150,9 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   const int G = cfg.group_size;
   const long long Cmax = cfg.max_budget;
   const bool write_scores = (cfg.flags & HE_FLAG_WRITE_SCORES) != 0;
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(rt_smem_raw) + 1023) & ~(uintptr_t)1023);
+  // rounded up to 1024 bytes by an offset from the array itself, so that the compiler still knows these are
+  // shared-memory addresses (a round trip through an integer would turn every access into a generic one)
+  unsigned char* smem = rt_smem_raw + ((1024u - (smem_u32(rt_smem_raw) & 1023u)) & 1023u);
   const RtLayout L = rt_layout(WORDS, a.smem_slots, G, !GLOBAL_TABLE, FP8);
   const int mp = GLOBAL_TABLE ? rt_mpitch(a.smem_slots, false) : kRtMaxSlots / kRtTile + 1;  // a constant for the smaller tables
   unsigned char* As = smem + L.a;
