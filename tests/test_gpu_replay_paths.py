@@ -27,6 +27,8 @@ shapes = [
     C["throughput_batch"].scaled(batch=2, budget_lo=130, budget_hi=300, group_size=3, hash_bits=40, decode_steps=2),
     C["llama3_8b_gqa"].scaled(batch=1, prompt_len=640, budget=129, hash_bits=4, decode_steps=2),
     C["llama3_8b_gqa"].scaled(batch=1, prompt_len=2100, budget=2049, hash_bits=8, decode_steps=2),
+    # four-bit codes over several tiles: most steps hit a stale tile maximum, so blocks are cut short after 64 repairs
+    C["llama3_8b_gqa"].scaled(batch=1, prompt_len=1800, budget=700, hash_bits=4, decode_steps=2),
 ]
 for w in shapes:
     case = Case(w)
