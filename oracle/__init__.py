@@ -51,6 +51,10 @@ def _load():
         lib.orc_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32]
         lib.orc_oneshot_codes.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, i32]
         lib.orc_oneshot_codes.restype = None
+        lib.orc_oneshot_l2.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, i32]
+        lib.orc_oneshot_l2.restype = None
+        lib.orc_attention_loss.argtypes = [vp, vp, vp, vp, vp, vp]
+        lib.orc_attention_loss.restype = None
         lib.orc_attend.argtypes = [vp, vp, vp, vp]
         lib.orc_attend.restype = None
         for f in (lib.orc_hash, lib.orc_reset, lib.orc_step_codes, lib.orc_step, lib.orc_prefill_codes, lib.orc_prefill):
@@ -151,6 +155,26 @@ class OracleCache:
         _load().orc_oneshot_codes(ctypes.byref(self._cfg), ctypes.byref(self._ca), _p(kcodes), _p(qcodes), _p(k), _p(v),
                                   _p(ks), _p(plen), Nmax, _p(sums), self.threads)
         return sums
+
+    def oneshot_l2(self, kcodes, k, v, prompt_len, want_norms=False):
+        """One-shot ranking by key L2 norm (the comparison policy the paper names); fills the cache with the kept tokens."""
+        Nmax = k.shape[2]
+        plen = np.ascontiguousarray(prompt_len, dtype=np.int32)
+        kcodes = np.ascontiguousarray(kcodes, dtype=np.uint32)
+        assert kcodes.shape == (self.B, self.H, Nmax, self.Wd) and k.strides == v.strides
+        ks = self._strides(k)
+        norms = np.zeros((self.B, self.H, Nmax), dtype=np.float32) if want_norms else None
+        _load().orc_oneshot_l2(ctypes.byref(self._cfg), ctypes.byref(self._ca), _p(kcodes), _p(k), _p(v), _p(ks), _p(plen), Nmax,
+                               _p(norms), self.threads)
+        return norms
+
+    def attention_loss(self, q, k_full):
+        """1 - attention mass of the cached tokens under q over all next_pos tokens seen. q [B, H*G, d] -> fp64 [B, H*G]."""
+        assert q.flags.c_contiguous and q.shape == (self.B, self.H * self.G, self.d)
+        ks = self._strides(k_full)
+        out = np.zeros((self.B, self.H * self.G), dtype=np.float64)
+        _load().orc_attention_loss(ctypes.byref(self._cfg), ctypes.byref(self._ca), _p(q), _p(k_full), _p(ks), _p(out))
+        return out
 
     def attend(self, q):
         """Eq. 1 over the compressed cache (Algorithm 1 line 6). q [B, H*G, d] -> fp64 [B, H*G, d]."""

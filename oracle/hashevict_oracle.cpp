@@ -347,6 +347,105 @@ extern "C" void orc_oneshot_codes(const orc_config* cfg, orc_cache* ca, const ui
   });
 }
 
+// Squared L2 norm of a key row in the precision that decides the L2 ranking: fp32, channels in ascending order, one
+// fused multiply-add per channel starting from 0 (the inputs are widened exactly).
+static inline float norm2_f32(const void* x, int dtype, int d) {
+  float acc = 0.0f;
+  for (int c = 0; c < d; ++c) {
+    const float xc = (float)load_elem(x, c, dtype);
+    acc = std::fmaf(xc, xc, acc);
+  }
+  return acc;
+}
+
+// The comparison policy the paper names (Section 1 / Section 4 setup: "dropping tokens based on the high L2 norms of
+// their key embeddings"; Appendix B calls its ranking "a low-to-high ordering of all L2 key norms"), as a one-shot
+// prompt-compression variant under the same boundary: tokens inside the protected windows first (token order), then
+// by squared key norm ascending, equal norms by token index; the first min(N, C) stay, stored in token order. Slot s
+// holds the s-th kept token: K, V, its Eq. 2 code (so that the cache remains a valid state for Algorithm 1), position,
+// score = -norm2. norms_out [B, Hkv, Nmax] (nullable) receives norm2 of every prompt key. The cache is reset first.
+extern "C" void orc_oneshot_l2(const orc_config* cfg, orc_cache* ca, const uint32_t* kcodes, const void* k, const void* v,
+                               const int64_t* kv_strides, const int32_t* prompt_len, int32_t max_prompt_len,
+                               float* norms_out, int32_t threads) {
+  const int Wd = words_of(cfg->hash_bits), d = cfg->head_dim, es = esize(cfg->dtype);
+  const int64_t units = (int64_t)cfg->batch * cfg->n_kv_heads, Nmax = max_prompt_len, Cmax = cfg->max_budget;
+  orc_reset(cfg, ca);
+  for_units(units, threads, [=](int64_t u) {
+    const int64_t s = u / cfg->n_kv_heads, h = u % cfg->n_kv_heads;
+    const int32_t C = ca->budget[s], N = prompt_len[s];
+    std::vector<float> nrm(N);
+    for (int32_t i = 0; i < N; ++i) {
+      const int64_t off = (s * kv_strides[0] + h * kv_strides[1] + (int64_t)i * kv_strides[2]) * es;
+      nrm[i] = norm2_f32((const char*)k + off, cfg->dtype, d);
+      if (norms_out) norms_out[u * Nmax + i] = nrm[i];
+    }
+    std::vector<int32_t> order(N);
+    for (int32_t i = 0; i < N; ++i) order[i] = i;
+    auto prot = [&](int32_t i) { return i < cfg->n_sink || i >= N - cfg->n_recent; };
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+      const bool pa = prot(a), pb = prot(b);
+      if (pa != pb) return pa;
+      if (pa) return a < b;
+      if (nrm[a] != nrm[b]) return nrm[a] < nrm[b];
+      return a < b;
+    });
+    const int32_t keep = N < C ? N : C;
+    std::vector<int32_t> kept(order.begin(), order.begin() + keep);
+    std::sort(kept.begin(), kept.end());
+    for (int32_t sl = 0; sl < keep; ++sl) {
+      const int32_t t = kept[sl];
+      const int64_t slot = u * Cmax + sl;
+      const int64_t off = (s * kv_strides[0] + h * kv_strides[1] + (int64_t)t * kv_strides[2]) * es;
+      std::memcpy((char*)ca->k_cache + slot * d * es, (const char*)k + off, (size_t)d * es);
+      std::memcpy((char*)ca->v_cache + slot * d * es, (const char*)v + off, (size_t)d * es);
+      for (int w = 0; w < Wd; ++w) ca->codes[slot * Wd + w] = kcodes[(u * Nmax + t) * Wd + w];
+      ca->pos[slot] = t;
+      ca->scores[slot] = -nrm[t];
+    }
+    ca->fill[u] = keep;
+    ca->next_pos[u] = N;
+  });
+}
+
+// Attention loss of a compressed cache (Section 4.6 / Appendix B: "the sum of the attention probabilities for the
+// evicted tokens. Or equivalently, 1 - the sum of the attention probabilities for the tokens in the compressed
+// cache"). For every unit and each of its G query heads, with a = softmax_p(q_g . k_p / sqrt(d)) over ALL n = next_pos
+// tokens seen so far (k_full strided [B, Hkv, n, d]):  loss = 1 - sum_{valid slots j} a[pos_j].  out [B, Hkv*G] fp64.
+// A unit that has seen no token gives 0.
+extern "C" void orc_attention_loss(const orc_config* cfg, const orc_cache* ca, const void* q, const void* k_full,
+                                   const int64_t* kv_strides, double* out) {
+  const int d = cfg->head_dim, G = cfg->group_size, es = esize(cfg->dtype);
+  const int64_t units = (int64_t)cfg->batch * cfg->n_kv_heads, Cmax = cfg->max_budget;
+  for (int64_t u = 0; u < units; ++u) {
+    const int64_t s = u / cfg->n_kv_heads, h = u % cfg->n_kv_heads;
+    const int n = ca->next_pos[u], fill = ca->fill[u];
+    for (int g = 0; g < G; ++g) {
+      const char* qg = (const char*)q + (u * G + g) * d * es;
+      if (n == 0) {
+        out[u * G + g] = 0.0;
+        continue;
+      }
+      std::vector<double> a(n);
+      double mx = -INFINITY;
+      for (int p = 0; p < n; ++p) {
+        const char* kp = (const char*)k_full + (s * kv_strides[0] + h * kv_strides[1] + (int64_t)p * kv_strides[2]) * es;
+        double dot = 0.0;
+        for (int c = 0; c < d; ++c) dot += load_elem(qg, c, cfg->dtype) * load_elem(kp, c, cfg->dtype);
+        a[p] = dot / std::sqrt((double)d);
+        if (a[p] > mx) mx = a[p];
+      }
+      double den = 0.0;
+      for (int p = 0; p < n; ++p) {
+        a[p] = std::exp(a[p] - mx);
+        den += a[p];
+      }
+      double keptsum = 0.0;
+      for (int j = 0; j < fill; ++j) keptsum += a[ca->pos[u * Cmax + j]] / den;
+      out[u * G + g] = 1.0 - keptsum;
+    }
+  }
+}
+
 // Eq. 1 over the compressed cache (Algorithm 1 line 6): for every unit and each of its G query heads,
 //   out[g] = sum_j softmax_j( q_g . K_j / sqrt(d) ) V_j   over the valid slots j < fill.
 // q: [B, Hkv*G, d] in the cache dtype; out: [B, Hkv*G, d] fp64. A unit with no valid slot gives zeros.

@@ -389,3 +389,81 @@ def test_oneshot_special_cases():
     assert sums[0, 0].tolist() == [G * b * (N - 1 - i) for i in range(N)]  # complementary codes: every bit differs
     # average G*b for all but the last token (0): the last token first, then the lowest indices
     assert oc.pos[0, 0].tolist() == [0, 1, 2, 3, N - 1]
+
+
+# ---------------------------------------------------------------- L2-norm ranking and attention loss (comparison policy, Section 4.6)
+
+def test_l2_ranking_norms_order_and_state():
+    rng = np.random.default_rng(3)
+    B, H, N, C, d, b = 2, 2, 41, 12, 16, 8
+    k = rng.standard_normal((B, H, N, d)).astype(np.float32)
+    v = rng.standard_normal((B, H, N, d)).astype(np.float32)
+    k[0, 0, 7] = k[0, 0, 3]  # equal norms: the lower index ranks first
+    k[1, 1, :, :] *= np.linspace(2.0, 0.5, N, dtype=np.float32)[:, None]  # norms fall with the position: the newest stay
+    kc = rng.integers(0, 256, size=(B, H, N, 1), dtype=np.uint32)
+    plen = np.array([N, 9], dtype=np.int32)
+    for n_sink, n_recent in [(0, 0), (2, 3)]:
+        oc = oracle.OracleCache(B, H, 1, d, b, C, [C, C], "f32", n_sink=n_sink, n_recent=n_recent)
+        norms = oc.oneshot_l2(kc, k, v, plen, want_norms=True)
+        for s in range(B):
+            n_tok = int(plen[s])
+            for h in range(H):
+                exact = (k[s, h, :n_tok].astype(np.float64) ** 2).sum(1)
+                np.testing.assert_allclose(norms[s, h, :n_tok], exact, rtol=2e-6)  # fp32 chain of 16 terms
+                prot = [i for i in range(n_tok) if i < n_sink or i >= n_tok - n_recent]
+                rest = sorted((i for i in range(n_tok) if i not in prot), key=lambda i: (norms[s, h, i], i))
+                keep = sorted((prot + rest)[:min(n_tok, C)])
+                fill = int(oc.fill[s, h])
+                assert oc.pos[s, h, :fill].tolist() == keep and oc.next_pos[s, h] == n_tok
+                for sl, t in enumerate(keep):
+                    assert np.array_equal(oc.k_cache[s, h, sl], k[s, h, t]) and oc.codes[s, h, sl, 0] == kc[s, h, t, 0]
+                    assert oc.scores[s, h, sl] == -norms[s, h, t]
+        if n_sink == 0:
+            assert oc.pos[1, 1, :9].tolist() == list(range(9))  # short prompt: everything stays
+    # the summation order is part of the definition: 2^12 squared, then sixteen ones, in fp32
+    x = np.zeros((1, 1, 2, 32), dtype=np.float32)
+    x[0, 0, 0, 0] = 4096.0
+    x[0, 0, 0, 1:17] = 1.0   # ascending chain: each +1 is lost against 2^24
+    x[0, 0, 1, 16] = 4096.0
+    x[0, 0, 1, 0:16] = 1.0   # the ones first: 16, then + 2^24 is exact
+    oc = oracle.OracleCache(1, 1, 1, 32, 8, 4, [4], "f32")
+    nn = oc.oneshot_l2(np.zeros((1, 1, 2, 1), dtype=np.uint32), x, x, [2], want_norms=True)
+    assert nn[0, 0].tolist() == [2.0 ** 24, 2.0 ** 24 + 16.0]
+
+
+def test_attention_loss_closed_forms_and_library_softmax():
+    import torch
+
+    w, W, K, Q, V, oc = run_tiny(0, 0, 2, 16, C=16, N=40, T=0, dtype="bf16")
+    q = np.ascontiguousarray(Q[:, :, 39])
+    oc.prefill(W, Q, K, V, np.array([40, 11], dtype=np.int32))
+    loss = oc.attention_loss(q, K)
+    Kd, qd = torch.from_numpy(wl.as_f64(w, K)), torch.from_numpy(wl.as_f64(w, q))
+    for s in range(2):
+        n = int(oc.next_pos[s, 0])
+        for h in range(w.n_kv_heads):
+            fill = int(oc.fill[s, h])
+            for g in range(2):
+                a = torch.softmax((Kd[s, h, :n] @ qd[s, h * 2 + g]) / np.sqrt(w.head_dim), dim=0).numpy()
+                want = 1.0 - a[oc.pos[s, h, :fill]].sum()
+                assert abs(loss[s, h * 2 + g] - want) < 1e-12
+    assert np.all(np.abs(loss[1]) < 1e-12)  # the second prompt fits its budget: nothing was dropped
+    assert np.all(loss[0] > 0) and np.all(loss[0] < 1)
+    # equal keys: uniform attention, the loss is the dropped fraction
+    oc2 = oracle.OracleCache(1, 1, 1, 8, 8, 4, [4], "f32")
+    kk = np.ones((1, 1, 10, 8), dtype=np.float32)
+    oc2.oneshot_l2(np.zeros((1, 1, 10, 1), dtype=np.uint32), kk, kk, [10])
+    out = oc2.attention_loss(np.full((1, 1, 8), 0.3, dtype=np.float32), kk)
+    assert abs(out[0, 0] - 0.6) < 1e-12
+    # one key carries all the attention: loss 0 if it is cached, 1 if it is not
+    kk[0, 0, 2] = 50.0   # huge norm: the L2 ranking drops it first
+    oc2.oneshot_l2(np.zeros((1, 1, 10, 1), dtype=np.uint32), kk, kk, [10])
+    assert 2 not in oc2.pos[0, 0].tolist()
+    assert oc2.attention_loss(np.ones((1, 1, 8), dtype=np.float32), kk)[0, 0] > 1 - 1e-12
+    # the opposite: a zero key (lowest norm, ranked first) under a query that scores every other key far below it
+    kk = np.full((1, 1, 10, 8), 3.0, dtype=np.float32)
+    kk[0, 0, 2] = 0.0
+    oc2.oneshot_l2(np.zeros((1, 1, 10, 1), dtype=np.uint32), kk, kk, [10])
+    assert 2 in oc2.pos[0, 0].tolist()
+    out = oc2.attention_loss(-np.ones((1, 1, 8), dtype=np.float32), kk)[0, 0]
+    assert 0 < out < 6 * np.exp(-24 / np.sqrt(8)) * 1.01  # six dropped keys, each e^(-24/sqrt 8) of the kept zero key
