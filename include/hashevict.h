@@ -182,6 +182,33 @@ int he_prefill_oneshot(const he_config* cfg, const he_cache* cache, const void* 
                        int32_t max_prompt_len, void* workspace, size_t workspace_bytes, long long* sums_out, void* stream);
 
 /*
+ * he_prefill_oneshot_l2 - the comparison policy the paper names (Section 1, Section 4 setup: dropping tokens by the
+ * high L2 norm of their key embeddings; Appendix B: "a low-to-high ordering of all L2 key norms") as a one-shot prompt
+ * compression under the same boundary. Not HashEvict: it is here so that both policies can be measured on the same
+ * cache layout. Order: protected tokens first (token order), then by squared key norm ascending, equal norms by
+ * token index; the first min(N, C) stay, stored in token order. The norm is taken in fp32 with channels in ascending
+ * order, one fused multiply-add per channel starting from 0 (this precision decides the ranking). Slot s holds the
+ * s-th kept token: K, V, its Eq. 2 code (the cache stays a valid state for he_decode_step), position, score = -norm2.
+ * No queries are read. workspace >= he_oneshot_workspace_bytes(cfg, max_prompt_len); max_prompt_len <= 32768;
+ * norms_out (device, nullable) [B, Hkv, max_prompt_len] fp32 receives norm2 of every prompt key.
+ */
+int he_prefill_oneshot_l2(const he_config* cfg, const he_cache* cache, const void* k, const void* v, const int64_t kv_strides[3],
+                          const int32_t* prompt_len, int32_t max_prompt_len, void* workspace, size_t workspace_bytes,
+                          float* norms_out, void* stream);
+
+/*
+ * he_attention_loss - attention loss of the compressed cache (Section 4.6, Appendix B): for every unit and each of its
+ * G query heads, out = sum of softmax_p(q . k_p / sqrt(d)) over the tokens p < next_pos that are NOT in the cache,
+ * i.e. 1 - the attention mass of the cached tokens, the softmax being over ALL next_pos tokens seen so far.
+ * q [B, Hkv*G, d] (cfg dtype, contiguous); k_full: every key seen so far, strided [B, Hkv, n, d] with element strides
+ * kv_strides (batch, head, token), n >= next_pos of every unit and n <= max_tokens; out [B, Hkv*G] fp32. The dropped
+ * mass is summed directly in fp32 (online maximum), so small losses keep their relative accuracy (about 1e-5). A unit
+ * that has seen no token gives 0. The cache is only read.
+ */
+int he_attention_loss(const he_config* cfg, const he_cache* cache, const void* q, const void* k_full,
+                      const int64_t kv_strides[3], int32_t max_tokens, float* out, void* stream);
+
+/*
  * he_prefill_compress_noalloc - he_prefill_compress for callers that cannot obtain device memory for the
  * prompt-code workspace. (The paper has no counterpart: this is a packaging variant, the computation and the
  * results are those of he_prefill_compress.)

@@ -36,7 +36,7 @@ class he_cache(ctypes.Structure):
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
     "he_decode_staging_bytes", "he_decode_step_host", "he_prefill_staging_bytes", "he_prefill_compress_host",
-    "he_prefill_compress_noalloc", "he_attend", "he_prefill_oneshot", "he_oneshot_workspace_bytes", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
+    "he_prefill_compress_noalloc", "he_attend", "he_prefill_oneshot", "he_oneshot_workspace_bytes", "he_prefill_oneshot_l2", "he_attention_loss", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
 )
 
 _lib = None
@@ -68,6 +68,8 @@ def lib():
     L.he_prefill_compress_host.argtypes = [cfgp, cap, vp, vp, vp, vp, i32, vp, vp, sz, vp]
     L.he_prefill_compress_noalloc.argtypes = [cfgp, cap, vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), vp, i32, vp]
     L.he_prefill_oneshot.argtypes = [cfgp, cap, vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), vp, i32, vp, sz, vp, vp]
+    L.he_prefill_oneshot_l2.argtypes = [cfgp, cap, vp, vp, ctypes.POINTER(i64), vp, i32, vp, sz, vp, vp]
+    L.he_attention_loss.argtypes = [cfgp, cap, vp, vp, ctypes.POINTER(i64), i32, vp, vp]
     L.he_oneshot_workspace_bytes.argtypes = [cfgp, i32]
     L.he_oneshot_workspace_bytes.restype = sz
     L.he_attend.argtypes = [cfgp, cap, vp, vp, vp]
@@ -213,6 +215,27 @@ class HashEvictCache:
         _check(lib().he_prefill_oneshot(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q), _ptr(k), _ptr(v),
                                         i64x3(*q.stride()[:3]), i64x3(*k.stride()[:3]), _ptr(prompt_len), nmax,
                                         _ptr(self._ws), self._ws.numel(), _ptr(sums_out), _stream(stream)))
+
+    def prefill_oneshot_l2(self, k, v, prompt_len, max_prompt_len=None, norms_out=None, stream=None):
+        """he_prefill_oneshot_l2: keep the min(N, C) prompt tokens with the lowest key L2 norm (the comparison policy)."""
+        nmax = k.shape[2] if max_prompt_len is None else max_prompt_len
+        need = lib().he_oneshot_workspace_bytes(ctypes.byref(self.cfg), nmax)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.k_cache.device)
+        assert k.stride(3) == 1 and k.stride() == v.stride()
+        i64x3 = ctypes.c_int64 * 3
+        _check(lib().he_prefill_oneshot_l2(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(k), _ptr(v), i64x3(*k.stride()[:3]),
+                                           _ptr(prompt_len), nmax, _ptr(self._ws), self._ws.numel(), _ptr(norms_out), _stream(stream)))
+
+    def attention_loss(self, q, k_full, out=None, stream=None):
+        """he_attention_loss: attention mass of the tokens that are no longer cached. q [B, H*G, d], k_full [B, H, n, d] -> fp32 [B, H*G]."""
+        if out is None:
+            out = torch.empty((self.B, self.H * self.G), dtype=torch.float32, device=self.k_cache.device)
+        assert k_full.stride(3) == 1
+        i64x3 = ctypes.c_int64 * 3
+        _check(lib().he_attention_loss(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q), _ptr(k_full), i64x3(*k_full.stride()[:3]),
+                                       k_full.shape[2], _ptr(out), _stream(stream)))
+        return out
 
     def prefill_compress_noalloc(self, q, k, v, prompt_len, max_prompt_len=None, stream=None):
         """he_prefill_compress_noalloc: same call, prompt codes go to the library's built-in scratch (no workspace,

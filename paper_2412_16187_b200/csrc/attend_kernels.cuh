@@ -335,4 +335,99 @@ __global__ void __launch_bounds__(kAttendThreads) attend_generic_kernel(const At
   attend_merge(part_ml, part_o, G, d, a.out + (size_t)unit * G * d);
 }
 
+// ------------------------------------------------------------------------------------------------ attention loss
+//
+// he_attention_loss (Section 4.6 / Appendix B): 1 - the attention mass of the cached tokens, for each query head, under
+// softmax(q . k_p / sqrt(d)) over ALL n = next_pos tokens seen so far. The dropped mass is summed directly (a token
+// is dropped when no valid slot holds its position: a bitmap in shared memory), so a small loss is not the
+// difference of two numbers close to one. One CTA per unit, a warp per token, online maximum as in he_attend.
+struct LossArgs {
+  he_config cfg;
+  he_cache ca;
+  const void* q;       // [B, Hkv*G, d]
+  const void* k_full;  // strided [B, Hkv, n, d]
+  long long s0, s1, s2;
+  float* out;          // [B, Hkv*G]
+};
+
+__global__ void __launch_bounds__(kAttendThreads) attention_loss_kernel(const LossArgs a) {
+  extern __shared__ __align__(16) float lsm_[];  // q as fp32 [G][d], partials [warps][G][3], bitmap of cached positions
+  const he_config& cfg = a.cfg;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long unit = (long long)blockIdx.y * cfg.n_kv_heads + blockIdx.x;
+  const int d = cfg.head_dim, G = cfg.group_size, es = esize_of(cfg.dtype);
+  const int n = a.ca.next_pos[unit], fill = a.ca.fill[unit];
+  float* qs = lsm_;
+  float* part = qs + G * d;
+  uint32_t* kept = reinterpret_cast<uint32_t*>(part + kAttendWarps * G * 3);
+  const int cpr = d * es / 16;
+  for (int idx = tid; idx < G * cpr; idx += kAttendThreads)
+    stage_chunk(qs + (idx / cpr) * d, static_cast<const char*>(a.q) + (unit * G + idx / cpr) * d * es, idx % cpr, cfg.dtype);
+  for (int i = tid; i < (n + 31) / 32; i += kAttendThreads) kept[i] = 0u;
+  __syncthreads();
+  for (int j = tid; j < fill; j += kAttendThreads) {
+    const int p = a.ca.pos[unit * cfg.max_budget + j];
+    if (p >= 0 && p < n) atomicOr(&kept[p >> 5], 1u << (p & 31));
+  }
+  __syncthreads();
+  const float scale = rsqrtf((float)d) * kLog2e;
+  const char* Kb = static_cast<const char*>(a.k_full) + ((long long)blockIdx.y * a.s0 + (long long)blockIdx.x * a.s1) * es;
+  float m[kMaxGroup], lall[kMaxGroup], ldrop[kMaxGroup];
+#pragma unroll
+  for (int g = 0; g < kMaxGroup; ++g) m[g] = -INFINITY, lall[g] = 0.f, ldrop[g] = 0.f;
+  const int per = (d + 31) / 32;
+  for (int p = warp; p < n; p += kAttendWarps) {
+    const char* kr = Kb + (long long)p * a.s2 * es;
+    float kv[kMaxDim / 32];
+#pragma unroll
+    for (int i = 0; i < kMaxDim / 32; ++i) {
+      const int c = lane + 32 * i;
+      kv[i] = (i < per && c < d) ? (cfg.dtype == HE_DTYPE_BF16 ? bf16_bits_to_f32(reinterpret_cast<const uint16_t*>(kr)[c])
+                                                                : reinterpret_cast<const float*>(kr)[c])
+                                 : 0.f;
+    }
+    const bool dropped = ((kept[p >> 5] >> (p & 31)) & 1u) == 0u;
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) {
+      if (g < G) {
+        float dot = 0.f;
+#pragma unroll
+        for (int i = 0; i < kMaxDim / 32; ++i) {
+          const int c = lane + 32 * i;
+          if (i < per && c < d) dot = fmaf(qs[g * d + c], kv[i], dot);
+        }
+        for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, off);
+        const float sc = dot * scale;
+        const float mn = fmaxf(m[g], sc);
+        const float corr = exp2f(m[g] - mn), w = exp2f(sc - mn);
+        lall[g] = lall[g] * corr + w;
+        ldrop[g] = ldrop[g] * corr + (dropped ? w : 0.f);
+        m[g] = mn;
+      }
+    }
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g)
+      if (g < G) {
+        part[(warp * G + g) * 3] = m[g];
+        part[(warp * G + g) * 3 + 1] = lall[g];
+        part[(warp * G + g) * 3 + 2] = ldrop[g];
+      }
+  }
+  __syncthreads();
+  if (tid < G) {
+    float M = -INFINITY;
+    for (int w = 0; w < kAttendWarps; ++w) M = fmaxf(M, part[(w * G + tid) * 3]);
+    float A = 0.f, D = 0.f;
+    for (int w = 0; w < kAttendWarps; ++w) {
+      const float mw = part[(w * G + tid) * 3];
+      const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
+      A += part[(w * G + tid) * 3 + 1] * f;
+      D += part[(w * G + tid) * 3 + 2] * f;
+    }
+    a.out[unit * G + tid] = A > 0.f ? D / A : 0.f;
+  }
+}
+
 }  // namespace he

@@ -513,9 +513,11 @@ namespace {
 // Shared body of he_prefill_compress (oneshot = false: Algorithm 1 replayed over the prompt) and he_prefill_oneshot
 // (oneshot = true: the averaged-Hamming ranking of Appendix C): validation, Eq. 2 on the prompt's keys and queries,
 // the selection kernel(s), the gather of the surviving K / V rows.
-int prefill_impl(bool oneshot, const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
+int prefill_impl(int variant /* 0: Algorithm 1, 1: averaged Hamming, 2: L2 norm */, const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
                  const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len, int32_t max_prompt_len,
-                 void* workspace, size_t workspace_bytes, long long* sums_out, void* stream) {
+                 void* workspace, size_t workspace_bytes, void* rank_out, void* stream) {
+  const bool oneshot = variant != 0;
+  if (variant == 2) q = k, q_strides = kv_strides;  // no queries in this policy: only the checks below look at them
   if (int rc = check_config(cfg, true)) return rc;
   if (int rc = check_cache(cache)) return rc;
   if (!q || !k || !v || !q_strides || !kv_strides || !prompt_len || !workspace)
@@ -560,6 +562,7 @@ int prefill_impl(bool oneshot, const he_config* cfg, const he_cache* cache, cons
   job.s1 = kv_strides[1];
   job.s2 = kv_strides[2];
   if (int rc = launch_hash(job, max_prompt_len, (int)units, st, &image_built)) return rc;
+  if (variant != 2) {
   job.x = q;
   job.out = qcodes;
   job.mode = 2;
@@ -569,6 +572,7 @@ int prefill_impl(bool oneshot, const he_config* cfg, const he_cache* cache, cons
   job.s1 = q_strides[1];
   job.s2 = q_strides[2];
   if (int rc = launch_hash(job, max_prompt_len, (int)units * G, st, &image_built)) return rc;
+  }
 
   // phase 2: the sequential replay of Algorithm 1 over the prompt, one CTA per unit
   int32_t* sched = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(qcodes) +
@@ -577,9 +581,20 @@ int prefill_impl(bool oneshot, const he_config* cfg, const he_cache* cache, cons
     if (units > 0x7FFFFFFF) return fail(HE_ERR_UNSUPPORTED, "too many units");
     char* extra = static_cast<char*>(workspace) + he_workspace_bytes(cfg, max_prompt_len);
     OneshotArgs oa{*cfg, *cache, kcodes, qcodes, prompt_len, max_prompt_len, reinterpret_cast<int32_t*>(extra),
-                   reinterpret_cast<unsigned long long*>(extra + align_up((size_t)units * max_prompt_len * 4, 256)), sums_out};
-    if (Wd == 1) oneshot_rank_kernel<1><<<(unsigned)units, kOneshotThreads, 0, st>>>(oa);
-    else oneshot_rank_kernel<2><<<(unsigned)units, kOneshotThreads, 0, st>>>(oa);
+                   reinterpret_cast<unsigned long long*>(extra + align_up((size_t)units * max_prompt_len * 4, 256)),
+                   variant == 1 ? static_cast<long long*>(rank_out) : nullptr};
+    if (variant == 2) {
+      if (units > 65535) return fail(HE_ERR_UNSUPPORTED, "more than 65535 units in one prefill call");
+      NormArgs na{*cfg, k, kv_strides[0], kv_strides[1], kv_strides[2], prompt_len, max_prompt_len, oa.sums, static_cast<float*>(rank_out)};
+      if (max_prompt_len > 0)
+        key_norms_kernel<<<dim3((unsigned)((max_prompt_len + kOneshotThreads - 1) / kOneshotThreads), (unsigned)units), kOneshotThreads, 0, st>>>(na);
+      HE_CUDA_CHECK(cudaGetLastError());
+      if (Wd == 1) oneshot_rank_kernel<1, 1><<<(unsigned)units, kOneshotThreads, 0, st>>>(oa);
+      else oneshot_rank_kernel<2, 1><<<(unsigned)units, kOneshotThreads, 0, st>>>(oa);
+    } else {
+      if (Wd == 1) oneshot_rank_kernel<1, 0><<<(unsigned)units, kOneshotThreads, 0, st>>>(oa);
+      else oneshot_rank_kernel<2, 0><<<(unsigned)units, kOneshotThreads, 0, st>>>(oa);
+    }
     HE_CUDA_CHECK(cudaGetLastError());
   } else {
     ReplayArgs ra{*cfg, *cache, kcodes, qcodes, prompt_len, max_prompt_len, cfg->max_budget, sched};
@@ -603,15 +618,22 @@ extern "C" {
 int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
                         const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len,
                         int32_t max_prompt_len, void* workspace, size_t workspace_bytes, void* stream) {
-  return prefill_impl(false, cfg, cache, q, k, v, q_strides, kv_strides, prompt_len, max_prompt_len, workspace, workspace_bytes,
+  return prefill_impl(0, cfg, cache, q, k, v, q_strides, kv_strides, prompt_len, max_prompt_len, workspace, workspace_bytes,
                       nullptr, stream);
 }
 
 int he_prefill_oneshot(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
                        const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len,
                        int32_t max_prompt_len, void* workspace, size_t workspace_bytes, long long* sums_out, void* stream) {
-  return prefill_impl(true, cfg, cache, q, k, v, q_strides, kv_strides, prompt_len, max_prompt_len, workspace, workspace_bytes,
+  return prefill_impl(1, cfg, cache, q, k, v, q_strides, kv_strides, prompt_len, max_prompt_len, workspace, workspace_bytes,
                       sums_out, stream);
+}
+
+int he_prefill_oneshot_l2(const he_config* cfg, const he_cache* cache, const void* k, const void* v, const int64_t kv_strides[3],
+                          const int32_t* prompt_len, int32_t max_prompt_len, void* workspace, size_t workspace_bytes,
+                          float* norms_out, void* stream) {
+  return prefill_impl(2, cfg, cache, nullptr, k, v, nullptr, kv_strides, prompt_len, max_prompt_len, workspace, workspace_bytes,
+                      norms_out, stream);
 }
 
 int he_prefill_compress_noalloc(const he_config* cfg, const he_cache* cache, const void* q, const void* k,
@@ -679,6 +701,27 @@ int he_attend(const he_config* cfg, const he_cache* cache, const void* q, float*
     if (int rc = set_smem(attend_generic_kernel, smem)) return rc;
     attend_generic_kernel<<<grid, kAttendThreads, smem, st>>>(a);
   }
+  HE_CUDA_CHECK(cudaGetLastError());
+  return HE_OK;
+}
+
+int he_attention_loss(const he_config* cfg, const he_cache* cache, const void* q, const void* k_full,
+                      const int64_t kv_strides[3], int32_t max_tokens, float* out, void* stream) {
+  if (int rc = check_config(cfg, true)) return rc;
+  if (int rc = check_cache(cache)) return rc;
+  if (!q || !k_full || !kv_strides || !out) return fail(HE_ERR_INVALID_ARG, "q, k_full, kv_strides or out is null");
+  if (!aligned16(q) || !aligned16(k_full)) return fail(HE_ERR_INVALID_ARG, "q and k_full must be 16-byte aligned");
+  if (max_tokens < 0) return fail(HE_ERR_INVALID_ARG, "max_tokens %d < 0", max_tokens);
+  const int es = esize_of(cfg->dtype);
+  for (int i = 0; i < 3; ++i)
+    if ((kv_strides[i] * es) % 16 != 0) return fail(HE_ERR_INVALID_ARG, "strides must keep every row 16-byte aligned");
+  if (cfg->batch > 65535) return fail(HE_ERR_UNSUPPORTED, "batch %d > 65535 in one call", cfg->batch);
+  const int G = cfg->group_size, d = cfg->head_dim;
+  const size_t smem = ((size_t)G * d + (size_t)kAttendWarps * G * 3) * sizeof(float) + ((size_t)max_tokens + 31) / 32 * 4 + 16;
+  if (smem > 200 * 1024) return fail(HE_ERR_UNSUPPORTED, "max_tokens %d does not fit the kernel's bitmap", max_tokens);
+  if (int rc = set_smem(attention_loss_kernel, smem)) return rc;
+  LossArgs a{*cfg, *cache, q, k_full, kv_strides[0], kv_strides[1], kv_strides[2], out};
+  attention_loss_kernel<<<dim3((unsigned)cfg->n_kv_heads, (unsigned)cfg->batch), kAttendThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
 }

@@ -33,7 +33,49 @@ constexpr int kOneshotThreads = 256;
 constexpr int kOneshotWarps = kOneshotThreads / 32;
 constexpr unsigned long long kOneshotRanked = 1ull << 57;  // set in the keys of tokens outside the protected windows
 
-template <int WORDS>
+// Squared L2 norm of every prompt key in the precision that decides the L2 ranking: fp32, channels in ascending order,
+// one fused multiply-add per channel starting from 0. One thread per row (the chain is sequential by definition);
+// the float's bit pattern goes to the `sums` scratch, which the ranking kernel reads as its sort key.
+struct NormArgs {
+  he_config cfg;
+  const void* k;
+  long long s0, s1, s2;  // element strides (batch, head, token)
+  const int32_t* prompt_len;
+  long long Nmax;
+  int32_t* norm_bits;  // scratch [units, Nmax]
+  float* norms_out;    // optional [units, Nmax]
+};
+
+__global__ void __launch_bounds__(kOneshotThreads) key_norms_kernel(const NormArgs a) {
+  const long long unit = blockIdx.y;
+  const int s = (int)(unit / a.cfg.n_kv_heads), h = (int)(unit % a.cfg.n_kv_heads);
+  const int i = blockIdx.x * kOneshotThreads + threadIdx.x;
+  if (i >= a.prompt_len[s]) return;
+  const int d = a.cfg.head_dim, es = esize_of(a.cfg.dtype);
+  const char* row = static_cast<const char*>(a.k) + (s * a.s0 + h * a.s1 + (long long)i * a.s2) * es;
+  float acc = 0.f;
+  for (int c0 = 0; c0 < d * es / 16; ++c0) {  // 16 bytes at a time: 8 bf16 or 4 fp32 channels
+    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(row) + c0);
+    const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (a.cfg.dtype == HE_DTYPE_BF16) {
+        const float lo = __uint_as_float(wv[k] << 16), hi = __uint_as_float(wv[k] & 0xFFFF0000u);
+        acc = fmaf(lo, lo, acc);
+        acc = fmaf(hi, hi, acc);
+      } else {
+        const float x = __uint_as_float(wv[k]);
+        acc = fmaf(x, x, acc);
+      }
+    }
+  }
+  a.norm_bits[unit * a.Nmax + i] = __float_as_int(acc);
+  if (a.norms_out != nullptr) a.norms_out[unit * a.Nmax + i] = acc;
+}
+
+// POLICY 0: averaged Hamming distance (Appendix C). POLICY 1: squared key norm, ascending (the comparison policy the
+// paper names); `sums` then holds the norms' bit patterns written by key_norms_kernel, qcodes is not read.
+template <int WORDS, int POLICY>
 __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const OneshotArgs a) {
   __shared__ int chunk_cnt[kOneshotWarps][32 * WORDS];
   __shared__ unsigned int hist[256];
@@ -55,6 +97,7 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
   unsigned long long* keys = a.keys + unit * a.Nmax;
 
   // ---- (1) S_i. Tokens are split into one contiguous chunk per warp; a lane counts the ones of its bits.
+  if (POLICY == 0) {
   const int chunk = (N + kOneshotWarps - 1) / kOneshotWarps;
   const int lo = min(N, warp * chunk), hi = min(N, lo + chunk);
   int cnt[WORDS];
@@ -93,6 +136,7 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
     }
   }
   __syncthreads();
+  }
 
   // ---- (2) keys: protected tokens sort first in token order, the others by average, then index
   for (int i = tid; i < N; i += kOneshotThreads) {
@@ -100,7 +144,9 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
     const int n = N - 1 - i;
     unsigned long long key = (unsigned long long)i;
     if (!prot) {
-      const unsigned long long q = n > 0 ? ((unsigned long long)(uint32_t)S[i] << 32) / (unsigned long long)n : 0ull;
+      unsigned long long q;
+      if (POLICY == 0) q = n > 0 ? ((unsigned long long)(uint32_t)S[i] << 32) / (unsigned long long)n : 0ull;
+      else q = (unsigned long long)(uint32_t)S[i];  // bits of a non-negative float order like the float
       key = kOneshotRanked | (q << 15) | (unsigned long long)i;
     }
     keys[i] = key;
@@ -158,7 +204,7 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
       for (int w = 0; w < WORDS; ++w) a.ca.codes[dst * WORDS + w] = kc_u[(long long)i * WORDS + w];
       a.ca.pos[dst] = i;
       const int n = N - 1 - i;
-      a.ca.scores[dst] = n > 0 ? -((float)S[i] / (float)n) : 0.f;
+      a.ca.scores[dst] = POLICY == 0 ? (n > 0 ? -((float)S[i] / (float)n) : 0.f) : -__int_as_float(S[i]);
       ++slot;
     }
   }
