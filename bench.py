@@ -419,6 +419,40 @@ def run_ours(args, w):
                                    "achieved": obytes / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
                                    "frac": obytes / (ms * 1e-3) / 1e9 / peak, "algorithmic_bytes_per_call": obytes}
 
+    if rank == 0 and not args.skip_oneshot:
+        # ---- secondary figure: attention loss (Section 4.6) of the three prompt-compression policies on this synthetic
+        # workload: mass of softmax(q K^T / sqrt(d)) over the whole prompt that falls on tokens no longer cached, for
+        # the first decode query of every head. Synthetic keys and queries: the numbers say nothing about a real model.
+        c0 = caches[0]
+        lo = torch.empty((B, H * G), dtype=torch.float32, device="cuda")
+        losses = {}
+        with torch.cuda.stream(stream):
+            for name, fill in (("algorithm_1", lambda: c0.prefill_compress(dQ, dK, dV, dplen, Nmax, workspace=ws, stream=stream)),
+                               ("oneshot_avg_hamming", lambda: c0.prefill_oneshot(dQ, dK, dV, dplen, Nmax, stream=stream)),
+                               ("l2_norm", lambda: c0.prefill_oneshot_l2(dK, dV, dplen, Nmax, stream=stream))):
+                fill()
+                c0.attention_loss(gq[0], dK, out=lo, stream=stream)
+                stream.synchronize()
+                losses[name] = float(lo.mean().item())
+            l0, l1, l2 = ev(), ev(), ev()
+            l0.record(stream)
+            for _ in range(4):
+                c0.attention_loss(gq[0], dK, out=lo, stream=stream)
+            l1.record(stream)
+            for _ in range(4):
+                c0.prefill_oneshot_l2(dK, dV, dplen, Nmax, stream=stream)
+            l2.record(stream)
+        torch.cuda.synchronize()
+        ms = l0.elapsed_time(l1) / 4
+        line["prefill_oneshot_l2"] = {"what": "he_prefill_oneshot_l2: keep the lowest key norms (comparison policy), per call",
+                                      "ms_per_call": l1.elapsed_time(l2) / 4,
+                                      "keys_per_s": float(plens.sum()) * H / (l1.elapsed_time(l2) / 4 * 1e-3)}
+        esz = 2 if w.dtype == "bf16" else 4
+        lbytes = float(plens.sum()) * H * d * esz
+        line["attention_loss"] = {"what": "he_attention_loss after each prompt-compression policy (mean over heads), synthetic data",
+                                  "mean_loss": losses, "ms_per_call": ms, "achieved_gbs": lbytes / (ms * 1e-3) / 1e9,
+                                  "frac": lbytes / (ms * 1e-3) / 1e9 / peak}
+
     if rank == 0:
         line["clocks"] = clocks
         if not args.skip_cpu_baseline and world == 1:

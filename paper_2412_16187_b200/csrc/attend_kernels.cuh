@@ -430,4 +430,115 @@ __global__ void __launch_bounds__(kAttendThreads) attention_loss_kernel(const Lo
   }
 }
 
+// The same for bf16 keys with d = 128 and G <= 8: scores of 16 tokens at a time as warp-level MMAs fed straight from
+// 16-byte global loads (the fragment scheme of attend_bf16_kernel), next group's rows requested before the current
+// group's arithmetic. Dynamic shared memory: partials [warps][G][3] floats, then the bitmap of cached positions.
+__global__ void __launch_bounds__(kAttendThreads) attention_loss_bf16_kernel(const LossArgs a) {
+  extern __shared__ __align__(16) float lsm_[];
+  constexpr int d = 128;
+  const he_config& cfg = a.cfg;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gid = lane >> 2, tig = lane & 3;
+  const long long unit = (long long)blockIdx.y * cfg.n_kv_heads + blockIdx.x;
+  const int G = cfg.group_size;
+  const int n = a.ca.next_pos[unit], fill = a.ca.fill[unit];
+  float* part = lsm_;
+  uint32_t* kept = reinterpret_cast<uint32_t*>(part + kAttendWarps * G * 3);
+  for (int i = tid; i < (n + 31) / 32; i += kAttendThreads) kept[i] = 0u;
+  __syncthreads();
+  for (int j = tid; j < fill; j += kAttendThreads) {
+    const int p = a.ca.pos[unit * cfg.max_budget + j];
+    if (p >= 0 && p < n) atomicOr(&kept[p >> 5], 1u << (p & 31));
+  }
+  __syncthreads();
+  uint32_t qf[8][2];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint4 t = make_uint4(0u, 0u, 0u, 0u);
+    if (gid < G) t = static_cast<const uint4*>(a.q)[(unit * G + gid) * (d / 8) + tig + 4 * c];
+    qf[2 * c][0] = t.x, qf[2 * c][1] = t.y, qf[2 * c + 1][0] = t.z, qf[2 * c + 1][1] = t.w;
+  }
+  const float scale = rsqrtf((float)d) * kLog2e;
+  const char* Kb = static_cast<const char*>(a.k_full) + ((long long)blockIdx.y * a.s0 + (long long)blockIdx.x * a.s1) * 2;
+  const int last = n - 1;
+  auto load_k = [&](int g0, uint4 (&kb)[2][4]) {  // rows past the end repeat the last row and are weighted by zero
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const uint4* row = reinterpret_cast<const uint4*>(Kb + (long long)min(g0 + gid + 8 * r, last) * a.s2 * 2);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) kb[r][c] = ldg_stream16(row + tig + 4 * c);
+    }
+  };
+  float m = -INFINITY, lall = 0.f, ldrop = 0.f;
+  uint4 kc[2][4], kn[2][4];
+  const int stride = 16 * kAttendWarps;
+  int g0 = 16 * warp;
+  if (g0 < n) load_k(g0, kc);
+  for (; g0 < n; g0 += stride) {
+    const bool more = g0 + stride < n;
+    if (more) load_k(g0 + stride, kn);
+    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      mma_bf16_m16n8k16(s0, qf[2 * c][0], 0u, qf[2 * c][1], 0u, kc[0][c].x, kc[0][c].y);
+      mma_bf16_m16n8k16(s1, qf[2 * c][0], 0u, qf[2 * c][1], 0u, kc[1][c].x, kc[1][c].y);
+      mma_bf16_m16n8k16(s0, qf[2 * c + 1][0], 0u, qf[2 * c + 1][1], 0u, kc[0][c].z, kc[0][c].w);
+      mma_bf16_m16n8k16(s1, qf[2 * c + 1][0], 0u, qf[2 * c + 1][1], 0u, kc[1][c].z, kc[1][c].w);
+    }
+    // this lane: head gid, tokens g0 + 2tig, + 1, + 8, + 9
+    const int j = g0 + 2 * tig;
+    const int tok[4] = {j, j + 1, j + 8, j + 9};
+    const float sc[4] = {s0[0], s0[1], s1[0], s1[1]};
+    float x[4];
+    bool dropped[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      x[e] = tok[e] < n ? sc[e] * scale : -INFINITY;
+      dropped[e] = tok[e] < n && ((kept[tok[e] >> 5] >> (tok[e] & 31)) & 1u) == 0u;
+    }
+    float gm = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+    gm = fmaxf(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, 1));
+    gm = fmaxf(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, 2));  // finite: token g0 exists
+    const float mn = fmaxf(m, gm);
+    const float corr = exp2f(m - mn);
+    float wa = 0.f, wd = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float w = exp2f(x[e] - mn);
+      wa += w;
+      wd += dropped[e] ? w : 0.f;
+    }
+    lall = lall * corr + wa;
+    ldrop = ldrop * corr + wd;
+    m = mn;
+    if (more) {
+#pragma unroll
+      for (int r = 0; r < 2; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) kc[r][c] = kn[r][c];
+    }
+  }
+  lall += __shfl_xor_sync(0xFFFFFFFFu, lall, 1);
+  lall += __shfl_xor_sync(0xFFFFFFFFu, lall, 2);
+  ldrop += __shfl_xor_sync(0xFFFFFFFFu, ldrop, 1);
+  ldrop += __shfl_xor_sync(0xFFFFFFFFu, ldrop, 2);
+  if (gid < G && tig == 0) {
+    part[(warp * G + gid) * 3] = m;
+    part[(warp * G + gid) * 3 + 1] = lall;
+    part[(warp * G + gid) * 3 + 2] = ldrop;
+  }
+  __syncthreads();
+  if (tid < G) {
+    float M = -INFINITY;
+    for (int w = 0; w < kAttendWarps; ++w) M = fmaxf(M, part[(w * G + tid) * 3]);
+    float A = 0.f, D = 0.f;
+    for (int w = 0; w < kAttendWarps; ++w) {
+      const float mw = part[(w * G + tid) * 3];
+      const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
+      A += part[(w * G + tid) * 3 + 1] * f;
+      D += part[(w * G + tid) * 3 + 2] * f;
+    }
+    a.out[unit * G + tid] = A > 0.f ? D / A : 0.f;
+  }
+}
+
 }  // namespace he

@@ -717,11 +717,18 @@ int he_attention_loss(const he_config* cfg, const he_cache* cache, const void* q
     if ((kv_strides[i] * es) % 16 != 0) return fail(HE_ERR_INVALID_ARG, "strides must keep every row 16-byte aligned");
   if (cfg->batch > 65535) return fail(HE_ERR_UNSUPPORTED, "batch %d > 65535 in one call", cfg->batch);
   const int G = cfg->group_size, d = cfg->head_dim;
-  const size_t smem = ((size_t)G * d + (size_t)kAttendWarps * G * 3) * sizeof(float) + ((size_t)max_tokens + 31) / 32 * 4 + 16;
+  const bool fast = cfg->dtype == HE_DTYPE_BF16 && d == 128 && getenv("HE_DISABLE_ATTEND_MMA") == nullptr;
+  const size_t smem = ((fast ? 0 : (size_t)G * d) + (size_t)kAttendWarps * G * 3) * sizeof(float) + ((size_t)max_tokens + 31) / 32 * 4 + 16;
   if (smem > 200 * 1024) return fail(HE_ERR_UNSUPPORTED, "max_tokens %d does not fit the kernel's bitmap", max_tokens);
-  if (int rc = set_smem(attention_loss_kernel, smem)) return rc;
   LossArgs a{*cfg, *cache, q, k_full, kv_strides[0], kv_strides[1], kv_strides[2], out};
-  attention_loss_kernel<<<dim3((unsigned)cfg->n_kv_heads, (unsigned)cfg->batch), kAttendThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  const dim3 grid((unsigned)cfg->n_kv_heads, (unsigned)cfg->batch);
+  if (fast) {
+    if (int rc = set_smem(attention_loss_bf16_kernel, smem)) return rc;
+    attention_loss_bf16_kernel<<<grid, kAttendThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  } else {
+    if (int rc = set_smem(attention_loss_kernel, smem)) return rc;
+    attention_loss_kernel<<<grid, kAttendThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  }
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
 }

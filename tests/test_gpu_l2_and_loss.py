@@ -75,8 +75,13 @@ def check_loss(case, q_np, k_full_np):
 
 
 @pytest.mark.parametrize("name", ["tiny", "llama2_7b_layer", "llama3_8b_gqa", "throughput_batch"])
-def test_attention_loss_after_each_policy(name):
+@pytest.mark.parametrize("path", ["default", "generic"])
+def test_attention_loss_after_each_policy(name, path, monkeypatch):
     w = PARITY_CASES[name]
+    if path == "generic":
+        if w.dtype != "bf16" or w.head_dim != 128:
+            pytest.skip("the default path is already the generic kernel")
+        monkeypatch.setenv("HE_DISABLE_ATTEND_MMA", "1")
     q = np.ascontiguousarray(wl.gen_decode_inputs(w, "q", 0, 1)[0])
     case = Case(w)
     case.prefill()  # Algorithm 1
