@@ -118,8 +118,10 @@ __device__ __forceinline__ uint16_t bf16_rne_bits(float f) {
   return (uint16_t)(u >> 16);
 }
 
-// One element of W -> its three bf16 terms at their places in the image (term-major, then 64-channel half, then the
-// [N rows x 128 bytes] K-major tile with the 128-byte swizzle).
+// One element of W -> its three bf16 terms at their places in the image: per 64-channel half one K-major operand of
+// 3N rows (term 1's N bit rows, then term 2's, then term 3's), 128 bytes per row with the 128-byte swizzle. The three
+// terms are thus three column groups of ONE MMA (N = 96 or 192): a third of the instructions, and the kernel is bound
+// by MMA issue.
 __device__ __forceinline__ void w_image_element(const float* W, int d, int b, int N, int idx, unsigned char* image) {
   const int c = idx / N, i = idx % N, KH = d / 64, tile_bytes = N * 128;
   const float w = i < b ? __ldg(W + (long long)c * b + i) : 0.f;
@@ -130,9 +132,9 @@ __device__ __forceinline__ void w_image_element(const float* W, int d, int b, in
   const uint16_t w3 = bf16_rne_bits(r2);
   const int kh = c / 64, kk = c % 64;
   const int off = (i / 8) * 1024 + (i % 8) * 128 + (((kk / 8) ^ (i % 8)) * 16) + (kk % 8) * 2;
-  *reinterpret_cast<uint16_t*>(image + (0 * KH + kh) * tile_bytes + off) = w1;
-  *reinterpret_cast<uint16_t*>(image + (1 * KH + kh) * tile_bytes + off) = w2;
-  *reinterpret_cast<uint16_t*>(image + (2 * KH + kh) * tile_bytes + off) = w3;
+  *reinterpret_cast<uint16_t*>(image + (kh * 3 + 0) * tile_bytes + off) = w1;
+  *reinterpret_cast<uint16_t*>(image + (kh * 3 + 1) * tile_bytes + off) = w2;
+  *reinterpret_cast<uint16_t*>(image + (kh * 3 + 2) * tile_bytes + off) = w3;
 }
 
 // The image in global memory, built once per call when the caller has scratch for it (kWImageBytes at most).
@@ -201,6 +203,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
                                                                      long long tiles_per_seg,
                                                                      const __grid_constant__ CUtensorMap tmap) {
   constexpr int N = 32 * WORDS;
+  constexpr int kAccCols = 3 * N;                          // one accumulator: the three terms side by side
+  constexpr int kTmemCols = 2 * kAccCols <= 256 ? 256 : 512;  // two accumulators, rounded up to a power of two
   extern __shared__ unsigned char tc_smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * kTcStages + 4];
   __shared__ uint32_t tmem_base_s;
@@ -240,7 +244,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 5) {  // tensor memory: two accumulators of N columns each -> 2N columns (a power of two >= 32)
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2 * N)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -320,7 +324,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
     // ------------------------------------------------------------------ MMA issue (one thread)
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) /* fp32 accumulate */ | (1u << 7) /* A bf16 */ | (1u << 10) /* B bf16 */ |
-                             ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kTcRows >> 4) << 24);
+                             ((uint32_t)(kAccCols >> 3) << 17) | ((uint32_t)(kTcRows >> 4) << 24);
       const uint64_t b_desc0 = umma_desc_k128(smem_u32(Bs));
       int it = 0;
       for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
@@ -333,24 +337,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
         // Descriptors differ only in their 14-bit start-address field, so each MMA's pair is the tile's base
         // descriptor plus a small constant: the issuing thread spends a few instructions per MMA, not dozens.
         const uint64_t a_desc0 = umma_desc_k128(smem_u32(As + s * a_stage_bytes));
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * N);
-        if (KH == 2) {
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
 #pragma unroll
-          for (int term = 2; term >= 0; --term)  // smallest term first
+        for (int kh = 0; kh < 2; ++kh) {
+          if (kh < KH) {
 #pragma unroll
-            for (int kh = 0; kh < 2; ++kh)
-#pragma unroll
-              for (int ks = 0; ks < 4; ++ks)  // K = 16 bf16 = 32 bytes per instruction inside the 128-byte swizzle span
-                tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)((kh * (kTcRows * 128) + ks * 32) >> 4),
-                            b_desc0 + (uint64_t)(((term * 2 + kh) * (N * 128) + ks * 32) >> 4), idesc,
-                            !(term == 2 && kh == 0 && ks == 0));
-        } else {
-#pragma unroll
-          for (int term = 2; term >= 0; --term)
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)((ks * 32) >> 4), b_desc0 + (uint64_t)((term * (N * 128) + ks * 32) >> 4), idesc,
-                          !(term == 2 && ks == 0));
+            for (int ks = 0; ks < 4; ++ks)  // K = 16 bf16 = 32 bytes per instruction inside the 128-byte swizzle span
+              tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)((kh * (kTcRows * 128) + ks * 32) >> 4),
+                          b_desc0 + (uint64_t)((kh * 3 * (N * 128) + ks * 32) >> 4), idesc, !(kh == 0 && ks == 0));
+          }
         }
         tc_commit(empty_bar(s));    // the stage may be refilled once these MMAs have read it
         tc_commit(tfull_bar(acc));  // and the accumulator is complete
@@ -369,12 +364,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
       uint32_t code[WORDS];
 #pragma unroll
       for (int w = 0; w < WORDS; ++w) {
-        uint32_t v[32];
-        tc_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * N + w * 32), v);
+        uint32_t v1[32], v2[32], v3[32];
+        const uint32_t base = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * kAccCols + w * 32);
+        tc_ld32(base, v1);
+        tc_ld32(base + N, v2);
+        tc_ld32(base + 2 * N, v3);
         tc_wait_ld();
         uint32_t word = 0u;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) word |= (__uint_as_float(v[i]) >= 0.f ? 1u : 0u) << i;
+        for (int i = 0; i < 32; ++i) {  // the three terms' partial sums, smallest term first
+          const float p = (__uint_as_float(v3[i]) + __uint_as_float(v2[i])) + __uint_as_float(v1[i]);
+          word |= (p >= 0.f ? 1u : 0u) << i;
+        }
         code[w] = word & word_mask(b, w);
       }
       tc_fence_before();
@@ -394,7 +395,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   __syncthreads();
   if (warp == 5) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * N) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
   if (tid == 0 && abort_flag) atomicAdd(&g_tc_error, 1);
   griddep_wait();  // no-op unless this kernel was launched programmatically behind another one
