@@ -157,8 +157,20 @@ struct TcTile {
 template <int WORDS>
 __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long long tiles_per_seg, TcTile* o,
                                         const int* s_len, const int* s_bud) {
-  const int seg = (int)(t / tiles_per_seg);
-  const long long ti = t % tiles_per_seg;
+  // 64-bit division is emulated and every role calls this once per tile: keep it to 32 bits whenever the counts fit
+  int seg;
+  long long ti;
+  if (job.mode == 0) {
+    seg = 0;
+    ti = t;
+  } else if (t < 0x7FFFFFFFll && tiles_per_seg < 0x7FFFFFFFll) {
+    const unsigned tt = (unsigned)t, tp = (unsigned)tiles_per_seg;
+    seg = (int)(tt / tp);
+    ti = (long long)(tt - (unsigned)seg * tp);
+  } else {
+    seg = (int)(t / tiles_per_seg);
+    ti = t % tiles_per_seg;
+  }
   long long r_begin, r_end;
   if (job.mode == 0) {
     o->base = static_cast<const char*>(job.x);
