@@ -31,6 +31,7 @@ struct OneshotArgs {
 
 constexpr int kOneshotThreads = 256;
 constexpr int kOneshotWarps = kOneshotThreads / 32;
+constexpr int kOneshotSub = 64;  // tokens staged per warp at a time
 constexpr unsigned long long kOneshotRanked = 1ull << 57;  // set in the keys of tokens outside the protected windows
 
 // Squared L2 norm of every prompt key in the precision that decides the L2 ranking: fp32, channels in ascending order,
@@ -78,6 +79,8 @@ __global__ void __launch_bounds__(kOneshotThreads) key_norms_kernel(const NormAr
 template <int WORDS, int POLICY>
 __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const OneshotArgs a) {
   __shared__ int chunk_cnt[kOneshotWarps][32 * WORDS];
+  __shared__ uint32_t qbuf[POLICY == 0 ? kOneshotWarps : 1][kOneshotSub * kMaxGroup * WORDS];  // staged query codes, per warp
+  __shared__ uint32_t kbuf[POLICY == 0 ? kOneshotWarps : 1][kOneshotSub * WORDS];              // staged key codes
   __shared__ unsigned int hist[256];
   __shared__ unsigned long long s_prefix;
   __shared__ int s_want;
@@ -96,46 +99,62 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
   int32_t* S = a.sums + unit * a.Nmax;
   unsigned long long* keys = a.keys + unit * a.Nmax;
 
-  // ---- (1) S_i. Tokens are split into one contiguous chunk per warp; a lane counts the ones of its bits.
+  // ---- (1) S_i. Tokens are split into one contiguous chunk per warp; a lane counts the ones of its bits. Codes go
+  // through a per-warp shared-memory buffer, kOneshotSub tokens at a time, so that global loads are coalesced and
+  // the per-token loop reads broadcast words instead of waiting on a dependent global load.
   if (POLICY == 0) {
-  const int chunk = (N + kOneshotWarps - 1) / kOneshotWarps;
-  const int lo = min(N, warp * chunk), hi = min(N, lo + chunk);
-  int cnt[WORDS];
+    uint32_t* qb = qbuf[warp];
+    uint32_t* kb = kbuf[warp];
+    const int chunk = (N + kOneshotWarps - 1) / kOneshotWarps;
+    const int lo = min(N, warp * chunk), hi = min(N, lo + chunk);
+    int cnt[WORDS];
 #pragma unroll
-  for (int w = 0; w < WORDS; ++w) cnt[w] = 0;
-  for (int j = lo; j < hi; ++j) {  // ones per bit over this warp's chunk
-    for (int g = 0; g < G; ++g) {
+    for (int w = 0; w < WORDS; ++w) cnt[w] = 0;
+    for (int j0 = lo; j0 < hi; j0 += kOneshotSub) {  // ones per bit over this warp's chunk
+      const int nt = min(kOneshotSub, hi - j0);
+      for (int x = lane; x < nt * GW; x += 32) qb[x] = __ldg(qc_u + (long long)j0 * GW + x);
+      __syncwarp();
+      for (int x = 0; x < nt * G; ++x) {
 #pragma unroll
-      for (int w = 0; w < WORDS; ++w) cnt[w] += (__ldg(qc_u + (long long)j * GW + g * WORDS + w) >> lane) & 1u;
+        for (int w = 0; w < WORDS; ++w) cnt[w] += (qb[x * WORDS + w] >> lane) & 1u;
+      }
+      __syncwarp();
     }
-  }
 #pragma unroll
-  for (int w = 0; w < WORDS; ++w) chunk_cnt[warp][w * 32 + lane] = cnt[w];
-  __syncthreads();
+    for (int w = 0; w < WORDS; ++w) chunk_cnt[warp][w * 32 + lane] = cnt[w];
+    __syncthreads();
 #pragma unroll
-  for (int w = 0; w < WORDS; ++w) {  // ones per bit over all later chunks
-    cnt[w] = 0;
-    for (int x = warp + 1; x < kOneshotWarps; ++x) cnt[w] += chunk_cnt[x][w * 32 + lane];
-  }
-  for (int i = hi - 1; i >= lo; --i) {  // cnt = ones per bit over the tokens j > i
-    const int m = (N - 1 - i) * G;
-    int term = 0;
-#pragma unroll
-    for (int w = 0; w < WORDS; ++w) {
-      const uint32_t hbit = (__ldg(kc_u + (long long)i * WORDS + w) >> lane) & 1u;
-      term += hbit ? m - cnt[w] : cnt[w];
+    for (int w = 0; w < WORDS; ++w) {  // ones per bit over all later chunks
+      cnt[w] = 0;
+      for (int x = warp + 1; x < kOneshotWarps; ++x) cnt[w] += chunk_cnt[x][w * 32 + lane];
     }
-    const int Si = __reduce_add_sync(0xFFFFFFFFu, term);
-    if (lane == 0) {
-      S[i] = Si;
-      if (a.sums_out != nullptr) a.sums_out[unit * a.Nmax + i] = Si;
-    }
-    for (int g = 0; g < G; ++g) {
+    for (int j1 = hi; j1 > lo; j1 -= kOneshotSub) {  // sub-chunks from the back; cnt = ones per bit over the tokens j > i
+      const int j0 = max(lo, j1 - kOneshotSub), nt = j1 - j0;
+      for (int x = lane; x < nt * GW; x += 32) qb[x] = __ldg(qc_u + (long long)j0 * GW + x);
+      for (int x = lane; x < nt * WORDS; x += 32) kb[x] = __ldg(kc_u + (long long)j0 * WORDS + x);
+      __syncwarp();
+      for (int t = nt - 1; t >= 0; --t) {
+        const int i = j0 + t;
+        const int m = (N - 1 - i) * G;
+        int term = 0;
 #pragma unroll
-      for (int w = 0; w < WORDS; ++w) cnt[w] += (__ldg(qc_u + (long long)i * GW + g * WORDS + w) >> lane) & 1u;
+        for (int w = 0; w < WORDS; ++w) {
+          const uint32_t hbit = (kb[t * WORDS + w] >> lane) & 1u;
+          term += hbit ? m - cnt[w] : cnt[w];
+        }
+        const int Si = __reduce_add_sync(0xFFFFFFFFu, term);
+        if (lane == (t & 31)) {  // spread the stores over the lanes
+          S[i] = Si;
+          if (a.sums_out != nullptr) a.sums_out[unit * a.Nmax + i] = Si;
+        }
+        for (int g = 0; g < G; ++g) {
+#pragma unroll
+          for (int w = 0; w < WORDS; ++w) cnt[w] += (qb[(t * G + g) * WORDS + w] >> lane) & 1u;
+        }
+      }
+      __syncwarp();
     }
-  }
-  __syncthreads();
+    __syncthreads();
   }
 
   // ---- (2) keys: protected tokens sort first in token order, the others by average, then index
