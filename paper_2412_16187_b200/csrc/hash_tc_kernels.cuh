@@ -63,6 +63,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// Bounded wait on two barriers at once: both are polled in the same loop, so their latencies overlap (one polling
+// round trip costs a couple of hundred cycles even when the phase has long completed).
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b,
+                                           volatile int* abort_flag) {
+  bool ok_a = false, ok_b = false;
+  for (uint32_t i = 0; i < kTcSpinLimit; ++i) {
+    if (!ok_a) ok_a = mbar_try_wait(bar_a, parity_a);
+    if (!ok_b) ok_b = mbar_try_wait(bar_b, parity_b);
+    if (ok_a && ok_b) return true;
+    if (*abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -343,8 +358,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
         TcTile tl;
         if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud)) continue;
         const int s = it % kTcStages, acc = it & 1;
-        if (!mbar_wait(tempty_bar(acc), ((it >> 1) & 1) ^ 1, &abort_flag)) break;  // epilogue has drained this accumulator
-        if (!mbar_wait(full_bar(s), (it / kTcStages) & 1, &abort_flag)) break;
+        // the epilogue has drained this accumulator and the stage's rows have landed
+        if (!mbar_wait2(tempty_bar(acc), ((it >> 1) & 1) ^ 1, full_bar(s), (it / kTcStages) & 1, &abort_flag)) break;
         tc_fence_after();
         // Descriptors differ only in their 14-bit start-address field, so each MMA's pair is the tile's base
         // descriptor plus a small constant: the issuing thread spends a few instructions per MMA, not dozens.

@@ -394,8 +394,8 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           const uint64_t a_desc0 = umma_desc_k128(smem_u32(As));
           for (int i = 0; i < ntile; ++i) {
             const int n = it + i, st = n % NSTAGE, ph = (n / NSTAGE) & 1;
-            if (!mbar_wait(tempty_bar(st), ph ^ 1, &abort_flag)) break;  // readers have drained this accumulator
-            if (!mbar_wait(full_bar(st), ph, &abort_flag)) break;
+            // the readers have drained this accumulator and the expanders have written this operand stage
+            if (!mbar_wait2(tempty_bar(st), ph ^ 1, full_bar(st), ph, &abort_flag)) break;
             tc_fence_after();
             const uint64_t b_desc0 = umma_desc_k128(smem_u32(Bs + st * ATOMS * kRtAtomBytes));
             const uint32_t d_tmem = tmem_base + (uint32_t)(st * kRtTile);
