@@ -166,14 +166,13 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
 
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };          // expanders -> MMA: operand stage s is written
-  auto empty_bar = [&](int s) { return bar0 + 8u * (NSTAGE + s); };       // MMA -> expanders: stage s has been read
   auto tfull_bar = [&](int x) { return bar0 + 8u * (2 * NSTAGE + x); };   // MMA -> readers: accumulator x is complete
+  auto empty_bar = tfull_bar;                                              // MMA -> expanders: stage x has been read (same event)
   auto tempty_bar = [&](int x) { return bar0 + 8u * (3 * NSTAGE + x); };  // readers -> MMA: accumulator x is drained
   if (tid == 0) {
     abort_flag = 0;
     for (int s = 0; s < NSTAGE; ++s) {
       mbar_init(full_bar(s), 128);
-      mbar_init(empty_bar(s), 1);
       mbar_init(tfull_bar(s), 1);
       mbar_init(tempty_bar(s), 4);
     }
@@ -408,8 +407,9 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
                 tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)(off >> 4), b_desc0 + (uint64_t)(off >> 4), idesc, ks > 0);
               }
             }
-            tc_commit(empty_bar(st));   // the operand stage may be rewritten once these MMAs have read it
-            tc_commit(tfull_bar(st));   // and the accumulator is complete
+            // one commit serves both consumers: when these MMAs are done the accumulator is complete (readers) and the
+            // operand stage may be rewritten (expanders); stage and accumulator share the index, so they share the barrier
+            tc_commit(tfull_bar(st));
           }
         }
       } else {
