@@ -491,7 +491,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
         bool scored = !(write_scores && t0 + rows == N);  // only the prompt's last step stores Eq. 5 scores
         int r = 0;
         while (r < rows) {
-          int status = 0;
+          int status = 0, kn_out = 0;
           for (; r < rows; ++r) {
             const int rn = r + 1 < rows ? r + 1 : r;  // the last step fetches its own row again (unused)
             const uint2 dd_n = *reinterpret_cast<const uint2*>(Dn + rn * kRtRows + 4 * lane);
@@ -509,6 +509,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             // best base slot: the tile maxima are upper bounds; one that points at an evicted slot needs a repair
             if (kb > kn && own_kb >= 0) {
               status = 1;
+              kn_out = kn;
               break;
             }
             if (!scored && r == rows - 1) {
@@ -543,11 +544,9 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             uint32_t qw[kMaxGroup * WORDS];
 #pragma unroll
             for (int i = 0; i < kMaxGroup * WORDS; ++i) qw[i] = i < GW ? qb[r * GW + i] : 0u;
-            const int k0 = (int)((dd.x & 0xFFFFu) << kRtKeyShift) + vb0;
-            const int k1 = (int)((dd.x >> 16) << kRtKeyShift) + vb1;
-            const int k2 = (int)((dd.y & 0xFFFFu) << kRtKeyShift) + vb2;
-            const int k3 = (int)((dd.y >> 16) << kRtKeyShift) + vb3;
-            const int kn = __reduce_max_sync(0xFFFFFFFFu, max(max(k0, k1), max(k2, k3)));
+            const int kn = kn_out;  // the step's best new entry, as the hot loop left it
+            // lane i keeps tile i's maximum for this step in a register (tables in shared memory: at most 32 tiles)
+            int mt = (!GLOBAL_TABLE && lane < nbase) ? Mx[r * mp + lane] : 0;
             for (int pass = 0; pass <= nbase; ++pass) {
               ++stale;
               const int cb = (kRtIdxMask - (kb & kRtIdxMask)) / kRtTile;
@@ -575,10 +574,15 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
                 km = max(km, ow[i] < 0 ? key : 0);
               }
               km = __reduce_max_sync(0xFFFFFFFFu, km);
-              Mx[r * mp + cb] = km;  // same value from every lane
-              int rowmax = lane < nbase ? Mx[r * mp + lane] : 0;
-              if (GLOBAL_TABLE)
-                for (int i = lane + 32; i < nbase; i += 32) rowmax = max(rowmax, Mx[r * mp + i]);
+              int rowmax;
+              if (GLOBAL_TABLE) {
+                Mx[r * mp + cb] = km;  // same value from every lane
+                rowmax = 0;
+                for (int i = lane; i < nbase; i += 32) rowmax = max(rowmax, Mx[r * mp + i]);
+              } else {
+                mt = lane == cb ? km : mt;
+                rowmax = mt;
+              }
               kb = __reduce_max_sync(0xFFFFFFFFu, rowmax);
               if (kb <= kn || owner[kRtIdxMask - (kb & kRtIdxMask)] < 0) break;
             }
