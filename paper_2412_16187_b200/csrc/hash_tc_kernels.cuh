@@ -138,7 +138,7 @@ __device__ __forceinline__ uint16_t bf16_rne_bits(float f) {
 // terms are thus three column groups of ONE MMA (N = 96 or 192): a third of the instructions, and the kernel is bound
 // by MMA issue.
 __device__ __forceinline__ void w_image_element(const float* W, int d, int b, int N, int idx, unsigned char* image) {
-  const int c = idx / N, i = idx % N, KH = d / 64, tile_bytes = N * 128;
+  const int c = idx / N, i = idx % N, tile_bytes = N * 128;
   const float w = i < b ? __ldg(W + (long long)c * b + i) : 0.f;
   const uint16_t w1 = bf16_rne_bits(w);
   const float r1 = w - bf16_bits_to_f32(w1);

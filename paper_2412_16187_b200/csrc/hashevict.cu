@@ -334,21 +334,21 @@ int launch_replay_reg(const ReplayArgs& a, long long units, cudaStream_t stream)
   return launch_replay_smem<WORDS, GT>(a, units, stream);
 }
 
-// Tensor-core replay: one persistent CTA per SM, for budgets up to 12288 slots without a protected window. Up to
-// 4096 slots the unit's tables sit in shared memory, beyond that they are the cache's own arrays.
-template <int WORDS, bool GLOBAL_TABLE, bool FP8>
+// Tensor-core replay: one persistent CTA per SM, for budgets up to 12288 slots. Up to 4096 slots the unit's tables sit in
+// shared memory (protected windows are handled there), beyond that they are the cache's own arrays.
+template <int WORDS, bool GLOBAL_TABLE, bool FP8, bool PROT = false>
 int launch_replay_tc_one(const ReplayArgs& a0, long long units, cudaStream_t stream) {
   ReplayArgs a = a0;
   a.smem_slots = (a.cfg.max_budget + kRtTile - 1) / kRtTile * kRtTile;
   const size_t smem = rt_layout(WORDS, a.smem_slots, a.cfg.group_size, !GLOBAL_TABLE, FP8).total;
-  if (int rc = set_smem(prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8>, smem)) return rc;
+  if (int rc = set_smem(prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8, PROT>, smem)) return rc;
   int sms = 0;
   if (int rc = sm_count(&sms)) return rc;
   const int nbins = sms < kMaxBins ? sms : kMaxBins;
   prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched);
   HE_CUDA_CHECK(cudaGetLastError());
   const long long grid = units < sms ? units : sms;
-  prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);
+  prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8, PROT><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
 }
@@ -357,7 +357,11 @@ int launch_replay_tc_one(const ReplayArgs& a0, long long units, cudaStream_t str
 template <int WORDS, bool GLOBAL_TABLE>
 int launch_replay_tc(const ReplayArgs& a, long long units, cudaStream_t stream) {
   const char* e = getenv("HE_TC_REPLAY_BF16");
-  if (a.cfg.group_size <= 7 && !(e && e[0] == '1')) return launch_replay_tc_one<WORDS, GLOBAL_TABLE, true>(a, units, stream);
+  const bool fp8 = a.cfg.group_size <= 7 && !(e && e[0] == '1');
+  if (!GLOBAL_TABLE && (a.cfg.n_sink > 0 || a.cfg.n_recent > 0))  // protected windows (shared-memory tables only)
+    return fp8 ? launch_replay_tc_one<WORDS, false, true, true>(a, units, stream)
+               : launch_replay_tc_one<WORDS, false, false, true>(a, units, stream);
+  if (fp8) return launch_replay_tc_one<WORDS, GLOBAL_TABLE, true>(a, units, stream);
   return launch_replay_tc_one<WORDS, GLOBAL_TABLE, false>(a, units, stream);
 }
 
@@ -372,8 +376,14 @@ int tc_replay_mode() {
 template <int WORDS>
 int launch_replay(const ReplayArgs& a, long long units, cudaStream_t stream) {
   const int mode = tc_replay_mode();
-  if (mode != 0 && a.cfg.max_budget <= kRtMaxSlotsGlobal && (mode == 2 || a.cfg.max_budget >= 512) && a.cfg.n_sink == 0 &&
-      a.cfg.n_recent == 0)
+  bool tc_ok = mode != 0 && a.cfg.max_budget <= kRtMaxSlotsGlobal && (mode == 2 || a.cfg.max_budget >= 512);
+  if (tc_ok && (a.cfg.n_sink > 0 || a.cfg.n_recent > 0)) {
+    // protected windows: tables in shared memory only, and every budget must leave an eligible slot at every step
+    // (n_sink + n_recent < C), which the host can only check on the caller's mirror of the budgets
+    tc_ok = a.cfg.max_budget <= kRtMaxSlots && a.cfg.n_recent < kRtRows && a.ca.budget_host != nullptr;
+    for (int s = 0; tc_ok && s < a.cfg.batch; ++s) tc_ok = a.ca.budget_host[s] > a.cfg.n_sink + a.cfg.n_recent;
+  }
+  if (tc_ok)
     return a.cfg.max_budget <= kRtMaxSlots ? launch_replay_tc<WORDS, false>(a, units, stream)
                                            : launch_replay_tc<WORDS, true>(a, units, stream);
   switch (a.cfg.group_size) {

@@ -125,7 +125,12 @@ __device__ __forceinline__ int rt_dist(const uint32_t* h, const uint32_t* q, int
 // the digits of the slot index), K = 32 per instruction: half the operand bytes and three instructions per tile
 // instead of five, four operand stages and four accumulators. The key columns are then
 //   A = [.. | 2^14 | 4096 | 256 | 16 | 1],  B = [.. | G K / 2 | idx >> 12 | (idx >> 8) & 15 | (idx >> 4) & 15 | idx & 15].
-template <int WORDS, bool GLOBAL_TABLE, bool FP8>
+// PROT (protected windows, Section 4 setup: the first n_sink prompt tokens and the n_recent newest tokens are never
+// evicted; requires every budget > n_sink + n_recent so that some slot is always eligible): nothing changes in the
+// operands. The resolver treats a best base slot that is not eligible at this step like a stale one (the repair
+// then takes the tile's best eligible slot), and a token that enters at step r joins the new entries only at step
+// r + n_recent + 1, when it stops being recent; until then, and in the next block, it cannot win.
+template <int WORDS, bool GLOBAL_TABLE, bool FP8, bool PROT = false>
 __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const ReplayArgs a) {
   constexpr int ATOMS = (WORDS == 2 && !FP8) ? 2 : 1;
   constexpr int KB = 32 * WORDS;             // code columns of the contraction
@@ -139,6 +144,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   __shared__ uint32_t tmem_base_s;
   __shared__ volatile int abort_flag;
   __shared__ int s_unit, s_done;
+  __shared__ uint16_t entry_slot[PROT ? kRtRows : 1];  // PROT: the slot each of the block's steps wrote to
   // four code bits -> four bf16 values: operand B takes +-1 (bit set: +1), operand A -+2^13 (bit set: -2^13)
   __shared__ uint2 s_lut_a[16], s_lut_b[16];
   // 8-bit operands: operand A is summed in f16 (-+2^13 per head) and keeps the high bytes (= e5m2); operand B takes a
@@ -484,7 +490,12 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
         int done = rows, stale = 0;
         uint2 dd = *reinterpret_cast<const uint2*>(Dn + 4 * lane);
         int kb = RB[0];
-        int own_kb = -1;  // nothing has been evicted yet
+        int own_kb = -1;  // nothing has been evicted yet; >= 0 means: this key's slot may not be taken, repair first
+        const int S = cfg.n_sink, Rn = cfg.n_recent;
+        if (PROT) {
+          const int p0 = pos_t[kRtIdxMask - (kb & kRtIdxMask)];
+          if (p0 < S || p0 >= t0 - Rn) own_kb = 0;
+        }
         uint32_t kc[WORDS];
 #pragma unroll
         for (int w = 0; w < WORDS; ++w) kc[w] = kb_codes[w];
@@ -497,6 +508,12 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             const uint2 dd_n = *reinterpret_cast<const uint2*>(Dn + rn * kRtRows + 4 * lane);
             const int kb_n = RB[rn];
             int own_n = owner[kRtIdxMask - (kb_n & kRtIdxMask)];
+            int act_slot = 0;
+            if (PROT) {  // eligibility of the next step's best base slot at that step; the slot of the entry that turns eligible
+              const int pn = pos_t[kRtIdxMask - (kb_n & kRtIdxMask)];
+              if (pn < S || pn >= t0 + r + 1 - Rn) own_n = 0;
+              if (Rn > 0 && r >= Rn) act_slot = entry_slot[r - Rn];
+            }
             uint32_t kc_n[WORDS];
 #pragma unroll
             for (int w = 0; w < WORDS; ++w) kc_n[w] = kb_codes[rn * WORDS + w];
@@ -520,8 +537,11 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             const int slot = kRtIdxMask - (best & kRtIdxMask);
             // a new entry that wins leaves: its lane recognises its own key (keys of resident entries are distinct,
             // absent ones are negative); then this step's token enters as entry r
-            const bool mine = lane == (r >> 2);
-            const int sel = r & 3, nv = kRtIdxMask - slot;
+            // (with protected windows: the entry of step r - n_recent, which is no longer recent from the next step on)
+            const int e_act = PROT ? r - Rn : r;
+            const bool mine = e_act >= 0 && lane == (e_act >> 2);
+            const int sel = e_act & 3, nv = kRtIdxMask - ((PROT && Rn > 0) ? act_slot : slot);
+            if (PROT) entry_slot[r] = (uint16_t)slot;
             vb0 = (mine && sel == 0) ? nv : (k0 == best ? kAbsent : vb0);
             vb1 = (mine && sel == 1) ? nv : (k1 == best ? kAbsent : vb1);
             vb2 = (mine && sel == 2) ? nv : (k2 == best ? kAbsent : vb2);
@@ -551,11 +571,15 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
               ++stale;
               const int cb = (kRtIdxMask - (kb & kRtIdxMask)) / kRtTile;
               uint32_t hw[kRtTile / 32][WORDS];
-              int ow[kRtTile / 32];
+              int ow[kRtTile / 32];  // < 0: the slot still holds its base token (and, PROT, that token is eligible now)
 #pragma unroll
               for (int i = 0; i < kRtTile / 32; ++i) {
                 const int j = cb * kRtTile + lane + 32 * i;  // below smem_slots: rows past the budget hold zeros
                 ow[i] = j < C ? (int)owner[j] : 0;
+                if (PROT && j < C) {
+                  const int pj = pos_t[j];
+                  if (pj < S || pj >= t0 + r - Rn) ow[i] = 0;
+                }
 #pragma unroll
                 for (int w = 0; w < WORDS; ++w) hw[i][w] = j < C ? table_word(j * WORDS + w) : 0u;
               }
@@ -584,7 +608,14 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
                 rowmax = mt;
               }
               kb = __reduce_max_sync(0xFFFFFFFFu, rowmax);
-              if (kb <= kn || owner[kRtIdxMask - (kb & kRtIdxMask)] < 0) break;
+              if (kb <= kn) break;
+              const int sb = kRtIdxMask - (kb & kRtIdxMask);
+              bool bad = owner[sb] >= 0;
+              if (PROT && !bad) {
+                const int pb = pos_t[sb];
+                bad = pb < S || pb >= t0 + r - Rn;
+              }
+              if (!bad) break;
             }
             own_kb = -1;  // exact for this step (or below the best new entry)
             if (stale >= kRtStaleLimit && r + 1 < rows && scored) {  // many repairs: this block ends with step r

@@ -1,7 +1,8 @@
 """Full-size cross-check of the replay implementations: at BASELINE sizes the oracle can only follow sampled units
 (tests/test_gpu_parity.py does that), so here the tensor-core replay (8-bit and bf16 operands) and the CUDA-core
 replay, each of which is checked against the oracle on smaller shapes, must leave bit-identical caches on the whole
-throughput_batch workload and on four layers of long_prefill (9830-slot budgets, tables in global memory)."""
+throughput_batch workload (also with the paper's protected windows) and on four layers of long_prefill (9830-slot
+budgets, tables in global memory)."""
 import hashlib
 import json
 import os
@@ -18,7 +19,8 @@ import sys, json, hashlib, numpy as np, torch
 sys.path.insert(0, %r)
 from paper_2412_16187_b200 import HashEvictCache, device_error_count, workloads as wl
 out = {}
-for name, w in (("throughput_batch", wl.CONFIGS["throughput_batch"]), ("long_prefill", wl.CONFIGS["long_prefill"].scaled(layers=4))):
+for name, w in (("throughput_batch", wl.CONFIGS["throughput_batch"]), ("long_prefill", wl.CONFIGS["long_prefill"].scaled(layers=4)),
+                ("throughput_batch_protected", wl.CONFIGS["throughput_batch"].scaled(batch=32, n_sink=4, n_recent=10))):
     B, H, G, d = w.n_seq, w.n_kv_heads, w.group_size, w.head_dim
     plens, Nmax = w.prompt_lens(), w.max_prompt_len
     def up(a):
@@ -29,7 +31,8 @@ for name, w in (("throughput_batch", wl.CONFIGS["throughput_batch"]), ("long_pre
         n = int(plens[s])
         dK[s, :, :n] = up(wl.gen_tokens(w, "k", s, 1, 0, n)[0]); dV[s, :, :n] = up(wl.gen_tokens(w, "v", s, 1, 0, n)[0])
         dQ[s, :, :n] = up(wl.gen_tokens(w, "q", s, 1, 0, n)[0])
-    c = HashEvictCache(B, H, G, d, w.hash_bits, w.budgets(), torch.from_numpy(wl.gen_W(w)), dtype=torch.bfloat16)
+    c = HashEvictCache(B, H, G, d, w.hash_bits, w.budgets(), torch.from_numpy(wl.gen_W(w)), dtype=torch.bfloat16, n_sink=w.n_sink,
+                       n_recent=w.n_recent)
     c.prefill_compress(dQ, dK, dV, torch.from_numpy(plens).cuda())
     torch.cuda.synchronize()
     h = hashlib.sha256()

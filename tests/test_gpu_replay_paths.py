@@ -1,7 +1,7 @@
 """The implementations of the prompt replay (tensor-core kernel with 8-bit or bf16 operands, CUDA-core kernels)
 against the oracle, each forced through the environment switches in a fresh process, on shapes that cover one-word and two-word codes, group
 sizes 1, 3 and 4, budgets that are not multiples of the 128-slot tile, ragged budgets, prompts that end inside a
-128-step block, prompts shorter than the budget, and keys with little variety (many equal distances, so the
+128-step block, prompts shorter than the budget, protected windows, and keys with little variety (many equal distances, so the
 lowest-slot rule and the repair of stale tile maxima are exercised)."""
 import os
 import subprocess
@@ -27,6 +27,14 @@ shapes = [
     C["throughput_batch"].scaled(batch=2, budget_lo=130, budget_hi=300, group_size=3, hash_bits=40, decode_steps=2),
     C["llama3_8b_gqa"].scaled(batch=1, prompt_len=640, budget=129, hash_bits=4, decode_steps=2),
     C["llama3_8b_gqa"].scaled(batch=1, prompt_len=2100, budget=2049, hash_bits=8, decode_steps=2),
+    # the paper's protected windows (first 4, newest 10), also with few-bit codes whose ties favour the sink slots, a window
+    # longer than a quarter of a block, and sinks without a recent window
+    PARITY_CASES["protected_gqa"].scaled(decode_steps=2),
+    PARITY_CASES["protected_tiny"].scaled(decode_steps=2),
+    C["llama3_8b_gqa"].scaled(batch=2, prompt_len=1500, budget=700, decode_steps=2, n_sink=4, n_recent=10),
+    C["llama3_8b_gqa"].scaled(batch=1, prompt_len=900, budget=260, hash_bits=4, decode_steps=2, n_sink=4, n_recent=10),
+    C["throughput_batch"].scaled(batch=2, budget_lo=200, budget_hi=400, decode_steps=2, n_sink=2, n_recent=45),
+    C["llama2_7b_layer"].scaled(prompt_len=700, budget=300, decode_steps=2, n_sink=7, n_recent=0),
     # four-bit codes over several tiles: most steps hit a stale tile maximum, so blocks are cut short after 64 repairs
     C["llama3_8b_gqa"].scaled(batch=1, prompt_len=1800, budget=700, hash_bits=4, decode_steps=2),
 ]
