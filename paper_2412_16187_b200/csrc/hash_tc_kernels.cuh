@@ -81,7 +81,7 @@ __device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t parity_a, ui
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// TMA tile copy global -> shared (no multicast), completion counted in bytes on `bar`
+// TMA tile copy global -> shared for this CTA alone, completion counted in bytes on `bar`
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tmap, int c0, int c1, int c2, int c3, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
