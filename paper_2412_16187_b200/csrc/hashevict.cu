@@ -335,7 +335,7 @@ int launch_replay_reg(const ReplayArgs& a, long long units, cudaStream_t stream)
 }
 
 // Tensor-core replay: one persistent CTA per SM, for budgets up to 12288 slots. Up to 4096 slots the unit's tables sit in
-// shared memory (protected windows are handled there), beyond that they are the cache's own arrays.
+// shared memory, beyond that they are the cache's own arrays.
 template <int WORDS, bool GLOBAL_TABLE, bool FP8, bool PROT = false>
 int launch_replay_tc_one(const ReplayArgs& a0, long long units, cudaStream_t stream) {
   ReplayArgs a = a0;
@@ -358,9 +358,9 @@ template <int WORDS, bool GLOBAL_TABLE>
 int launch_replay_tc(const ReplayArgs& a, long long units, cudaStream_t stream) {
   const char* e = getenv("HE_TC_REPLAY_BF16");
   const bool fp8 = a.cfg.group_size <= 7 && !(e && e[0] == '1');
-  if (!GLOBAL_TABLE && (a.cfg.n_sink > 0 || a.cfg.n_recent > 0))  // protected windows (shared-memory tables only)
-    return fp8 ? launch_replay_tc_one<WORDS, false, true, true>(a, units, stream)
-               : launch_replay_tc_one<WORDS, false, false, true>(a, units, stream);
+  if (a.cfg.n_sink > 0 || a.cfg.n_recent > 0)  // protected windows
+    return fp8 ? launch_replay_tc_one<WORDS, GLOBAL_TABLE, true, true>(a, units, stream)
+               : launch_replay_tc_one<WORDS, GLOBAL_TABLE, false, true>(a, units, stream);
   if (fp8) return launch_replay_tc_one<WORDS, GLOBAL_TABLE, true>(a, units, stream);
   return launch_replay_tc_one<WORDS, GLOBAL_TABLE, false>(a, units, stream);
 }
@@ -378,9 +378,10 @@ int launch_replay(const ReplayArgs& a, long long units, cudaStream_t stream) {
   const int mode = tc_replay_mode();
   bool tc_ok = mode != 0 && a.cfg.max_budget <= kRtMaxSlotsGlobal && (mode == 2 || a.cfg.max_budget >= 512);
   if (tc_ok && (a.cfg.n_sink > 0 || a.cfg.n_recent > 0)) {
-    // protected windows: tables in shared memory only, and every budget must leave an eligible slot at every step
-    // (n_sink + n_recent < C), which the host can only check on the caller's mirror of the budgets
-    tc_ok = a.cfg.max_budget <= kRtMaxSlots && a.cfg.n_recent < kRtRows && a.ca.budget_host != nullptr;
+    // protected windows: every budget must leave an eligible slot at every step (n_sink + n_recent < C), which the host
+    // can only check on the caller's mirror of the budgets; with the tables in global memory the kernel tracks the
+    // recent tokens in a 32-entry ring
+    tc_ok = a.cfg.n_recent <= (a.cfg.max_budget <= kRtMaxSlots ? kRtRows - 1 : 32) && a.ca.budget_host != nullptr;
     for (int s = 0; tc_ok && s < a.cfg.batch; ++s) tc_ok = a.ca.budget_host[s] > a.cfg.n_sink + a.cfg.n_recent;
   }
   if (tc_ok)

@@ -240,8 +240,17 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
       for (int w = 0; w < WORDS; ++w) codes_t[j * WORDS + w] = j < fill0 ? __ldg(kc_u + (long long)j * WORDS + w) : 0u;
       pos_t[j] = j < fill0 ? j : -1;
     }
+    // PROT with the tables in global memory: positions are too far away for the resolver's step-ahead checks, so warp 0
+    // keeps the slots of the 32 newest tokens in a register ring (lane l: the newest token congruent to l mod 32; the
+    // first C tokens sit in slot = position) and sinks are recognised by their slot (they never leave slots 0..n_sink-1).
+    int myring = -1;
+    if (PROT && GLOBAL_TABLE) {
+      const int pl = fill0 - 1 - ((fill0 - 1 - lane) & 31);
+      myring = pl >= 0 ? pl : -1;
+    }
     // A table word as the latest step left it (global tables: read past L1, which other warps' stores do not update)
     auto table_word = [&](int idx) -> uint32_t { return GLOBAL_TABLE ? __ldcg(codes_t + idx) : codes_t[idx]; };
+    auto table_pos = [&](int j) -> int { return GLOBAL_TABLE ? __ldcg(pos_t + j) : pos_t[j]; };
     __syncthreads();
     bool aborted = false;
     const int GW = G * WORDS;
@@ -492,10 +501,17 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
         int kb = RB[0];
         int own_kb = -1;  // nothing has been evicted yet; >= 0 means: this key's slot may not be taken, repair first
         const int S = cfg.n_sink, Rn = cfg.n_recent;
-        if (PROT) {
-          const int p0 = pos_t[kRtIdxMask - (kb & kRtIdxMask)];
-          if (p0 < S || p0 >= t0 - Rn) own_kb = 0;
-        }
+        // Is the token in `slot` protected at step t? With the ring: `first` = 1 leaves out the token of step t - 1, whose
+        // slot is not in the ring yet when the check runs one step ahead (the caller patches that case itself).
+        auto protected_at = [&](int slot, int t, int first) -> bool {
+          if (GLOBAL_TABLE) {
+            const int k = (t - 1 - lane) & 31;
+            return slot < S || __any_sync(0xFFFFFFFFu, myring == slot && k >= first && k < Rn);
+          }
+          const int p = pos_t[slot];
+          return p < S || p >= t - Rn;
+        };
+        if (PROT && protected_at(kRtIdxMask - (kb & kRtIdxMask), t0, 0)) own_kb = 0;
         uint32_t kc[WORDS];
 #pragma unroll
         for (int w = 0; w < WORDS; ++w) kc[w] = kb_codes[w];
@@ -510,8 +526,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             int own_n = owner[kRtIdxMask - (kb_n & kRtIdxMask)];
             int act_slot = 0;
             if (PROT) {  // eligibility of the next step's best base slot at that step; the slot of the entry that turns eligible
-              const int pn = pos_t[kRtIdxMask - (kb_n & kRtIdxMask)];
-              if (pn < S || pn >= t0 + r + 1 - Rn) own_n = 0;
+              if (protected_at(kRtIdxMask - (kb_n & kRtIdxMask), t0 + r + 1, 1)) own_n = 0;
               if (Rn > 0 && r >= Rn) act_slot = entry_slot[r - Rn];
             }
             uint32_t kc_n[WORDS];
@@ -542,6 +557,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             const bool mine = e_act >= 0 && lane == (e_act >> 2);
             const int sel = e_act & 3, nv = kRtIdxMask - ((PROT && Rn > 0) ? act_slot : slot);
             if (PROT) entry_slot[r] = (uint16_t)slot;
+            if (PROT && GLOBAL_TABLE && lane == ((t0 + r) & 31)) myring = slot;
             vb0 = (mine && sel == 0) ? nv : (k0 == best ? kAbsent : vb0);
             vb1 = (mine && sel == 1) ? nv : (k1 == best ? kAbsent : vb1);
             vb2 = (mine && sel == 2) ? nv : (k2 == best ? kAbsent : vb2);
@@ -577,7 +593,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
                 const int j = cb * kRtTile + lane + 32 * i;  // below smem_slots: rows past the budget hold zeros
                 ow[i] = j < C ? (int)owner[j] : 0;
                 if (PROT && j < C) {
-                  const int pj = pos_t[j];
+                  const int pj = table_pos(j);
                   if (pj < S || pj >= t0 + r - Rn) ow[i] = 0;
                 }
 #pragma unroll
@@ -612,7 +628,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
               const int sb = kRtIdxMask - (kb & kRtIdxMask);
               bool bad = owner[sb] >= 0;
               if (PROT && !bad) {
-                const int pb = pos_t[sb];
+                const int pb = table_pos(sb);
                 bad = pb < S || pb >= t0 + r - Rn;
               }
               if (!bad) break;
@@ -626,6 +642,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
 #pragma unroll
               for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
               pos_t[slot] = t0 + r;
+              if (PROT && GLOBAL_TABLE && lane == ((t0 + r) & 31)) myring = slot;
               done = r + 1;
               break;
             }

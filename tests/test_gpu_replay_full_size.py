@@ -20,7 +20,8 @@ sys.path.insert(0, %r)
 from paper_2412_16187_b200 import HashEvictCache, device_error_count, workloads as wl
 out = {}
 for name, w in (("throughput_batch", wl.CONFIGS["throughput_batch"]), ("long_prefill", wl.CONFIGS["long_prefill"].scaled(layers=4)),
-                ("throughput_batch_protected", wl.CONFIGS["throughput_batch"].scaled(batch=32, n_sink=4, n_recent=10))):
+                ("throughput_batch_protected", wl.CONFIGS["throughput_batch"].scaled(batch=32, n_sink=4, n_recent=10)),
+                ("long_prefill_protected", wl.CONFIGS["long_prefill"].scaled(layers=2, n_sink=4, n_recent=10))):
     B, H, G, d = w.n_seq, w.n_kv_heads, w.group_size, w.head_dim
     plens, Nmax = w.prompt_lens(), w.max_prompt_len
     def up(a):

@@ -35,6 +35,10 @@ shapes = [
     C["llama3_8b_gqa"].scaled(batch=1, prompt_len=900, budget=260, hash_bits=4, decode_steps=2, n_sink=4, n_recent=10),
     C["throughput_batch"].scaled(batch=2, budget_lo=200, budget_hi=400, decode_steps=2, n_sink=2, n_recent=45),
     C["llama2_7b_layer"].scaled(prompt_len=700, budget=300, decode_steps=2, n_sink=7, n_recent=0),
+    # budgets above 4096 slots (tables in global memory), plain and with protected windows up to the 32-token ring
+    C["long_prefill"].scaled(layers=1, n_kv_heads=2, prompt_len=7000, budget=4500, decode_steps=2),
+    C["long_prefill"].scaled(layers=1, n_kv_heads=2, prompt_len=7000, budget=4500, decode_steps=2, n_sink=4, n_recent=10),
+    C["long_prefill"].scaled(layers=1, n_kv_heads=1, prompt_len=6000, budget=4200, hash_bits=8, decode_steps=2, n_sink=3, n_recent=32),
     # four-bit codes over several tiles: most steps hit a stale tile maximum, so blocks are cut short after 64 repairs
     C["llama3_8b_gqa"].scaled(batch=1, prompt_len=1800, budget=700, hash_bits=4, decode_steps=2),
 ]
