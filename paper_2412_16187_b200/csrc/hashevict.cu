@@ -365,8 +365,10 @@ int launch_replay_tc(const ReplayArgs& a, long long units, cudaStream_t stream) 
   return launch_replay_tc_one<WORDS, GLOBAL_TABLE, false>(a, units, stream);
 }
 
-// HE_TC_REPLAY=0 keeps the replay on the CUDA-core kernels, =1 sends every eligible shape to the tensor-core kernel;
-// unset, the tensor-core kernel takes budgets from 512 slots up (below that a block of 128 steps no longer pays).
+// HE_TC_REPLAY=0 keeps the replay on the CUDA-core kernels, =1 sends every eligible shape to the tensor-core kernel.
+// Unset: the tensor-core kernel runs one unit per SM at about 400 cycles per step whatever the budget, the register
+// kernel several units per SM at a cost that grows with the budget; measured on B200 (512 units, b = 64, G = 4) they
+// cross between 1024 and 1280 slots, and with no more units than SMs already around 512 slots.
 int tc_replay_mode() {
   const char* e = getenv("HE_TC_REPLAY");
   if (!tc_enabled() || (e && e[0] == '0')) return 0;
@@ -376,7 +378,10 @@ int tc_replay_mode() {
 template <int WORDS>
 int launch_replay(const ReplayArgs& a, long long units, cudaStream_t stream) {
   const int mode = tc_replay_mode();
-  bool tc_ok = mode != 0 && a.cfg.max_budget <= kRtMaxSlotsGlobal && (mode == 2 || a.cfg.max_budget >= 512);
+  int sms = 0;
+  if (int rc = sm_count(&sms)) return rc;
+  const int min_budget = units <= sms ? 512 : 1152;
+  bool tc_ok = mode != 0 && a.cfg.max_budget <= kRtMaxSlotsGlobal && (mode == 2 || a.cfg.max_budget >= min_budget);
   if (tc_ok && (a.cfg.n_sink > 0 || a.cfg.n_recent > 0)) {
     // protected windows: every budget must leave an eligible slot at every step (n_sink + n_recent < C), which the host
     // can only check on the caller's mirror of the budgets; with the tables in global memory the kernel tracks the
