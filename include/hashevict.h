@@ -77,7 +77,9 @@ typedef struct he_cache {
   const int32_t* budget_host; /* optional HOST copy of budget ([B]), or NULL. When given (and B <= 1024)
                                  he_decode_step passes the budgets in the kernel parameters, which saves the
                                  kernel one dependent device read before it can start streaming the code table.
-                                 Must hold the same values as `budget`. */
+                                 With protected windows (n_sink or n_recent > 0) he_prefill_compress also needs it to
+                                 check that every budget exceeds n_sink + n_recent before it picks its faster replay
+                                 kernel; without it the call is correct but slower. Must hold the same values as `budget`. */
   uint32_t* step_scratch;     /* optional device buffer of he_step_scratch_bytes(cfg) bytes, or NULL. When given and
                                  a step has at least 16384 new rows (B * Hkv * (G + 1)), he_decode_step first hashes
                                  all of them with the bulk projection kernels into this buffer and the per-unit
