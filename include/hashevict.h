@@ -199,6 +199,18 @@ int he_prefill_oneshot_l2(const he_config* cfg, const he_cache* cache, const voi
                           float* norms_out, void* stream);
 
 /*
+ * he_decode_step_l2 - one decoding step of the same comparison policy under the boundary of he_decode_step: the new
+ * token always enters; while a unit's cache is full, the resident token with the highest squared key norm leaves
+ * (lowest slot on equal norms; protected windows and the "if no slot is eligible, all are" rule as in
+ * he_decode_step). It relies on scores[j] = -norm2 of the key in slot j, as he_prefill_oneshot_l2 and this call leave
+ * them; mixing it with he_decode_step on one cache is not meaningful. The slot's code is set to zero. k, v:
+ * [B, Hkv, d] contiguous device rows; victim_out [B, Hkv] (required), evicted_pos_out [B, Hkv] (nullable, -1 while
+ * appending). No queries are read.
+ */
+int he_decode_step_l2(const he_config* cfg, const he_cache* cache, const void* k, const void* v, int32_t* victim_out,
+                      int32_t* evicted_pos_out, void* stream);
+
+/*
  * he_attention_loss - attention loss of the compressed cache (Section 4.6, Appendix B): for every unit and each of its
  * G query heads, out = sum of softmax_p(q . k_p / sqrt(d)) over the tokens p < next_pos that are NOT in the cache,
  * i.e. 1 - the attention mass of the cached tokens, the softmax being over ALL next_pos tokens seen so far.

@@ -53,6 +53,8 @@ def _load():
         lib.orc_oneshot_codes.restype = None
         lib.orc_oneshot_l2.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, i32]
         lib.orc_oneshot_l2.restype = None
+        lib.orc_step_l2.argtypes = [vp, vp, vp, vp, vp, vp, i32]
+        lib.orc_step_l2.restype = None
         lib.orc_attention_loss.argtypes = [vp, vp, vp, vp, vp, vp]
         lib.orc_attention_loss.restype = None
         lib.orc_attend.argtypes = [vp, vp, vp, vp]
@@ -167,6 +169,14 @@ class OracleCache:
         _load().orc_oneshot_l2(ctypes.byref(self._cfg), ctypes.byref(self._ca), _p(kcodes), _p(k), _p(v), _p(ks), _p(plen), Nmax,
                                _p(norms), self.threads)
         return norms
+
+    def step_l2(self, k, v):
+        """One decoding step of the L2-norm comparison policy. k / v [B, H, d]. Returns victim, evicted_pos."""
+        victim = np.zeros((self.B, self.H), dtype=np.int32)
+        evicted = np.zeros((self.B, self.H), dtype=np.int32)
+        assert k.flags.c_contiguous and v.flags.c_contiguous
+        _load().orc_step_l2(ctypes.byref(self._cfg), ctypes.byref(self._ca), _p(k), _p(v), _p(victim), _p(evicted), self.threads)
+        return victim, evicted
 
     def attention_loss(self, q, k_full):
         """1 - attention mass of the cached tokens under q over all next_pos tokens seen. q [B, H*G, d] -> fp64 [B, H*G]."""

@@ -407,6 +407,49 @@ extern "C" void orc_oneshot_l2(const orc_config* cfg, orc_cache* ca, const uint3
   });
 }
 
+// One decoding step of the L2-norm comparison policy under the same boundary as Algorithm 1: the new token always
+// enters; while the cache is full the resident token with the HIGHEST squared key norm leaves (lowest slot on equal
+// norms; protected windows as in Algorithm 1, ignored for a step in which no slot is eligible). It relies on
+// scores[j] = -norm2 of the key in slot j, which orc_oneshot_l2 and this function maintain; the code of the slot is
+// set to zero (this policy has no use for it). k / v: [B, Hkv, d].
+extern "C" void orc_step_l2(const orc_config* cfg, orc_cache* ca, const void* k, const void* v, int32_t* victim_out,
+                            int32_t* evicted_pos_out, int32_t threads) {
+  const int Wd = words_of(cfg->hash_bits), d = cfg->head_dim, es = esize(cfg->dtype);
+  const int64_t units = (int64_t)cfg->batch * cfg->n_kv_heads, Cmax = cfg->max_budget;
+  for_units(units, threads, [=](int64_t u) {
+    const int32_t C = ca->budget[u / cfg->n_kv_heads];
+    float* scores = ca->scores + u * Cmax;
+    int32_t* pos = ca->pos + u * Cmax;
+    const int32_t fill = ca->fill[u], t = ca->next_pos[u];
+    const char* kr = (const char*)k + u * d * es;
+    const char* vr = (const char*)v + u * d * es;
+    int32_t slot = fill, evicted = -1;
+    if (fill >= C) {
+      slot = -1;
+      for (int pass = 0; pass < 2 && slot < 0; ++pass) {  // second pass: nothing was eligible, so everything is
+        float worst = 0.0f;
+        for (int32_t j = 0; j < fill; ++j) {
+          const bool eligible = pass == 1 || (pos[j] >= cfg->n_sink && pos[j] < t - cfg->n_recent);
+          if (eligible && (slot < 0 || scores[j] < worst)) {
+            worst = scores[j];
+            slot = j;
+          }
+        }
+      }
+      evicted = pos[slot];
+    }
+    std::memcpy((char*)ca->k_cache + (u * Cmax + slot) * d * es, kr, (size_t)d * es);
+    std::memcpy((char*)ca->v_cache + (u * Cmax + slot) * d * es, vr, (size_t)d * es);
+    for (int w = 0; w < Wd; ++w) ca->codes[(u * Cmax + slot) * Wd + w] = 0u;
+    scores[slot] = -norm2_f32(kr, cfg->dtype, d);
+    pos[slot] = t;
+    ca->next_pos[u] = t + 1;
+    ca->fill[u] = fill < C ? fill + 1 : fill;
+    if (victim_out) victim_out[u] = slot;
+    if (evicted_pos_out) evicted_pos_out[u] = evicted;
+  });
+}
+
 // Attention loss of a compressed cache (Section 4.6 / Appendix B: "the sum of the attention probabilities for the
 // evicted tokens. Or equivalently, 1 - the sum of the attention probabilities for the tokens in the compressed
 // cache"). For every unit and each of its G query heads, with a = softmax_p(q_g . k_p / sqrt(d)) over ALL n = next_pos

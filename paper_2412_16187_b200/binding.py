@@ -36,7 +36,7 @@ class he_cache(ctypes.Structure):
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
     "he_decode_staging_bytes", "he_decode_step_host", "he_prefill_staging_bytes", "he_prefill_compress_host",
-    "he_prefill_compress_noalloc", "he_attend", "he_prefill_oneshot", "he_oneshot_workspace_bytes", "he_prefill_oneshot_l2", "he_attention_loss", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
+    "he_prefill_compress_noalloc", "he_attend", "he_prefill_oneshot", "he_oneshot_workspace_bytes", "he_prefill_oneshot_l2", "he_attention_loss", "he_decode_step_l2", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
 )
 
 _lib = None
@@ -70,6 +70,7 @@ def lib():
     L.he_prefill_oneshot.argtypes = [cfgp, cap, vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), vp, i32, vp, sz, vp, vp]
     L.he_prefill_oneshot_l2.argtypes = [cfgp, cap, vp, vp, ctypes.POINTER(i64), vp, i32, vp, sz, vp, vp]
     L.he_attention_loss.argtypes = [cfgp, cap, vp, vp, ctypes.POINTER(i64), i32, vp, vp]
+    L.he_decode_step_l2.argtypes = [cfgp, cap, vp, vp, vp, vp, vp]
     L.he_oneshot_workspace_bytes.argtypes = [cfgp, i32]
     L.he_oneshot_workspace_bytes.restype = sz
     L.he_attend.argtypes = [cfgp, cap, vp, vp, vp]
@@ -226,6 +227,14 @@ class HashEvictCache:
         i64x3 = ctypes.c_int64 * 3
         _check(lib().he_prefill_oneshot_l2(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(k), _ptr(v), i64x3(*k.stride()[:3]),
                                            _ptr(prompt_len), nmax, _ptr(self._ws), self._ws.numel(), _ptr(norms_out), _stream(stream)))
+
+    def decode_step_l2(self, k, v, victim_out=None, evicted_pos_out=None, stream=None):
+        """he_decode_step_l2: one step of the L2-norm comparison policy. k / v [B, H, d]. Returns victim_out [B, H]."""
+        if victim_out is None:
+            victim_out = torch.empty((self.B, self.H), dtype=torch.int32, device=self.k_cache.device)
+        _check(lib().he_decode_step_l2(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(k), _ptr(v), _ptr(victim_out),
+                                       _ptr(evicted_pos_out), _stream(stream)))
+        return victim_out
 
     def attention_loss(self, q, k_full, out=None, stream=None):
         """he_attention_loss: attention mass of the tokens that are no longer cached. q [B, H*G, d], k_full [B, H, n, d] -> fp32 [B, H*G]."""

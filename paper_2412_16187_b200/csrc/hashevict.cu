@@ -721,6 +721,20 @@ int he_attend(const he_config* cfg, const he_cache* cache, const void* q, float*
   return HE_OK;
 }
 
+int he_decode_step_l2(const he_config* cfg, const he_cache* cache, const void* k, const void* v, int32_t* victim_out,
+                      int32_t* evicted_pos_out, void* stream) {
+  if (int rc = check_config(cfg, true)) return rc;
+  if (int rc = check_cache(cache)) return rc;
+  if (!k || !v || !victim_out) return fail(HE_ERR_INVALID_ARG, "k, v or victim_out is null");
+  if (!aligned16(k) || !aligned16(v)) return fail(HE_ERR_INVALID_ARG, "k, v must be 16-byte aligned");
+  if (cfg->batch > 65535) return fail(HE_ERR_UNSUPPORTED, "batch %d > 65535 in one decode call", cfg->batch);
+  if (cfg->max_budget > 0xFFFFFF) return fail(HE_ERR_UNSUPPORTED, "max_budget %d too large", cfg->max_budget);
+  StepL2Args a{*cfg, *cache, k, v, victim_out, evicted_pos_out};
+  decode_step_l2_kernel<<<dim3((unsigned)cfg->n_kv_heads, (unsigned)cfg->batch), kStepL2Threads, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  HE_CUDA_CHECK(cudaGetLastError());
+  return HE_OK;
+}
+
 int he_attention_loss(const he_config* cfg, const he_cache* cache, const void* q, const void* k_full,
                       const int64_t kv_strides[3], int32_t max_tokens, float* out, void* stream) {
   if (int rc = check_config(cfg, true)) return rc;

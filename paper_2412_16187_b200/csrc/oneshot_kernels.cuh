@@ -239,4 +239,86 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
   }
 }
 
+// he_decode_step_l2: one decoding step of the L2-norm comparison policy, one CTA per unit. scores[j] = -norm2 of the
+// key in slot j (kept by he_prefill_oneshot_l2 and by this kernel), so the victim is the eligible slot with the lowest
+// score, lowest slot on equal scores; if no slot is eligible, all are. The new key's norm is the same sequential fp32
+// chain as in key_norms_kernel (thread 0), computed while the others scan.
+struct StepL2Args {
+  he_config cfg;
+  he_cache ca;
+  const void* k;  // [B, Hkv, d]
+  const void* v;
+  int32_t* victim_out;
+  int32_t* evicted_pos_out;
+};
+
+constexpr int kStepL2Threads = 128;
+
+__global__ void __launch_bounds__(kStepL2Threads) decode_step_l2_kernel(const StepL2Args a) {
+  __shared__ unsigned long long wbest[2][kStepL2Threads / 32];
+  __shared__ float s_norm;
+  const he_config& cfg = a.cfg;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long unit = (long long)blockIdx.y * cfg.n_kv_heads + blockIdx.x;
+  const int d = cfg.head_dim, es = esize_of(cfg.dtype), Wd = (cfg.hash_bits + 31) / 32;
+  const long long Cmax = cfg.max_budget;
+  const int C = min(a.ca.budget[blockIdx.y], (int)Cmax);
+  const int fill = a.ca.fill[unit], t = a.ca.next_pos[unit];
+  const char* kr = static_cast<const char*>(a.k) + unit * d * es;
+  const char* vr = static_cast<const char*>(a.v) + unit * d * es;
+  if (tid == 0) {
+    float acc = 0.f;
+    for (int c = 0; c < d; ++c) {
+      const float x = cfg.dtype == HE_DTYPE_BF16 ? bf16_bits_to_f32(reinterpret_cast<const uint16_t*>(kr)[c])
+                                                 : reinterpret_cast<const float*>(kr)[c];
+      acc = fmaf(x, x, acc);
+    }
+    s_norm = acc;
+  }
+  int slot = fill;
+  if (fill >= C) {
+    // key = bits of norm2 (a non-negative float: ordered like its bits) above the inverted slot index
+    unsigned long long best_all = 0ull, best_el = 0ull;
+    const float* sc = a.ca.scores + unit * Cmax;
+    const int32_t* pp = a.ca.pos + unit * Cmax;
+    for (int j = tid; j < fill; j += kStepL2Threads) {
+      const unsigned long long key =
+          ((unsigned long long)__float_as_uint(-sc[j]) << 24) | (unsigned long long)(0xFFFFFF - j) | (1ull << 60);
+      best_all = max(best_all, key);
+      const int p = pp[j];
+      if (p >= cfg.n_sink && p < t - cfg.n_recent) best_el = max(best_el, key);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      best_all = max(best_all, __shfl_xor_sync(0xFFFFFFFFu, best_all, o));
+      best_el = max(best_el, __shfl_xor_sync(0xFFFFFFFFu, best_el, o));
+    }
+    if (lane == 0) wbest[0][warp] = best_all, wbest[1][warp] = best_el;
+    __syncthreads();
+    unsigned long long fa = 0ull, fe = 0ull;
+    for (int w = 0; w < kStepL2Threads / 32; ++w) fa = max(fa, wbest[0][w]), fe = max(fe, wbest[1][w]);
+    const unsigned long long fin = fe != 0ull ? fe : fa;
+    slot = 0xFFFFFF - (int)(fin & 0xFFFFFFull);
+  } else {
+    __syncthreads();
+  }
+  const long long dst = unit * Cmax + slot;
+  for (int i = tid; i < 2 * (d * es / 16); i += kStepL2Threads) {
+    const int half = d * es / 16;
+    const bool is_k = i < half;
+    const uint4 row = __ldg(reinterpret_cast<const uint4*>(is_k ? kr : vr) + (is_k ? i : i - half));
+    reinterpret_cast<uint4*>(static_cast<char*>(is_k ? a.ca.k_cache : a.ca.v_cache) + dst * d * es)[is_k ? i : i - half] = row;
+  }
+  if (tid == 0) {
+    int ev = -1;
+    if (fill >= C) ev = a.ca.pos[dst];
+    a.ca.pos[dst] = t;
+    a.ca.scores[dst] = -s_norm;
+    for (int w = 0; w < Wd; ++w) a.ca.codes[dst * Wd + w] = 0u;
+    if (fill < C) a.ca.fill[unit] = fill + 1;
+    a.ca.next_pos[unit] = t + 1;
+    a.victim_out[unit] = slot;
+    if (a.evicted_pos_out != nullptr) a.evicted_pos_out[unit] = ev;
+  }
+}
+
 }  // namespace he

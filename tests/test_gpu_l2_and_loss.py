@@ -108,3 +108,35 @@ def test_attention_loss_is_zero_when_nothing_was_dropped_and_on_empty_caches():
     out = case.gpu.attention_loss(to_dev(q, w), case.dK)
     torch.cuda.synchronize()
     assert not out.cpu().numpy().any()  # every token is still cached
+
+
+@pytest.mark.parametrize("name", ["tiny", "llama3_8b_gqa", "throughput_batch", "protected_gqa"])
+def test_l2_decode_steps_match_oracle(name):
+    w = PARITY_CASES[name]
+    case = run_l2(w)
+    steps = 12
+    dk, dv = wl.gen_decode_inputs(w, "k", 0, steps), wl.gen_decode_inputs(w, "v", 0, steps)
+    dk[5] = dk[2]  # a repeated key: equal norms, the lower slot must leave first when both are candidates
+    gk, gv = to_dev(dk, w), to_dev(dv, w)
+    victim = torch.empty((w.n_seq, w.n_kv_heads), dtype=torch.int32, device="cuda")
+    evicted = torch.empty_like(victim)
+    for i in range(steps):
+        case.gpu.decode_step_l2(gk[i], gv[i], victim, evicted)
+        torch.cuda.synchronize()
+        ovic, oev = case.orc.step_l2(np.ascontiguousarray(dk[i]), np.ascontiguousarray(dv[i]))
+        assert np.array_equal(victim.cpu().numpy(), ovic), f"victims differ at step {i}"
+        assert np.array_equal(evicted.cpu().numpy(), oev), f"evicted positions differ at step {i}"
+    case.compare_state()
+
+
+def test_l2_decode_from_an_empty_cache_appends_then_evicts():
+    w = PARITY_CASES["tiny"]
+    case = Case(w)
+    steps = int(w.budgets().max()) + 9
+    dk, dv = wl.gen_decode_inputs(w, "k", 0, steps), wl.gen_decode_inputs(w, "v", 0, steps)
+    gk, gv = to_dev(dk, w), to_dev(dv, w)
+    for i in range(steps):
+        vic = case.gpu.decode_step_l2(gk[i], gv[i])
+        ovic, _ = case.orc.step_l2(np.ascontiguousarray(dk[i]), np.ascontiguousarray(dv[i]))
+        assert np.array_equal(vic.cpu().numpy(), ovic)
+    case.compare_state()

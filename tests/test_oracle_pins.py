@@ -467,3 +467,35 @@ def test_attention_loss_closed_forms_and_library_softmax():
     assert 2 in oc2.pos[0, 0].tolist()
     out = oc2.attention_loss(-np.ones((1, 1, 8), dtype=np.float32), kk)[0, 0]
     assert 0 < out < 6 * np.exp(-24 / np.sqrt(8)) * 1.01  # six dropped keys, each e^(-24/sqrt 8) of the kept zero key
+
+
+def test_l2_decode_steps_keep_the_lowest_norms_and_the_newest_token():
+    rng = np.random.default_rng(9)
+    B, H, d, C, T = 1, 2, 16, 6, 30
+    for n_sink, n_recent in [(0, 0), (1, 2)]:
+        oc = oracle.OracleCache(B, H, 1, d, 8, C, [C], "f32", n_sink=n_sink, n_recent=n_recent)
+        ks = rng.standard_normal((T, B, H, d)).astype(np.float32) * rng.uniform(0.2, 3.0, size=(T, 1, H, 1)).astype(np.float32)
+        ks[11] = ks[7]  # equal norms: the lower slot leaves first
+        resident = [dict() for _ in range(H)]  # slot -> (token, norm2), replayed in Python
+        for t in range(T):
+            victim, evicted = oc.step_l2(np.ascontiguousarray(ks[t]), np.ascontiguousarray(-ks[t]))
+            for h in range(H):
+                n2 = np.float32(0)
+                for c in range(d):
+                    n2 = np.float32(np.float64(ks[t, 0, h, c]) ** 2 + np.float64(n2))  # one rounding per channel, ascending
+                res = resident[h]
+                if len(res) < C:
+                    slot, gone = len(res), -1
+                else:
+                    elig = [j for j in res if res[j][0] >= n_sink and res[j][0] < t - n_recent] or list(res)
+                    slot = min(elig, key=lambda j: (-res[j][1], j))
+                    gone = res[slot][0]
+                assert victim[0, h] == slot and evicted[0, h] == gone
+                res[slot] = (t, n2)
+                assert oc.pos[0, h, slot] == t and oc.scores[0, h, slot] == -n2  # the newest token is always resident
+                assert np.array_equal(oc.k_cache[0, h, slot], ks[t, 0, h]) and np.array_equal(oc.v_cache[0, h, slot], -ks[t, 0, h])
+        if (n_sink, n_recent) == (0, 0):  # what is left: the newest token and the C - 1 lowest norms before it
+            for h in range(H):
+                n2 = (ks[:T - 1, 0, h].astype(np.float64) ** 2).sum(1)
+                want = set(np.argsort(n2, kind="stable")[:C - 1].tolist()) | {T - 1}
+                assert set(oc.pos[0, h].tolist()) == want
