@@ -59,3 +59,52 @@ def test_replay_implementations_agree_at_full_size():
     ref = run({"HE_TC_REPLAY": "0"})
     assert run({"HE_TC_REPLAY": "1"}) == ref
     assert run({"HE_TC_REPLAY": "1", "HE_TC_REPLAY_BF16": "1"}) == ref
+
+
+RANDOM_SCRIPT = r"""
+import sys, json, hashlib, numpy as np, torch
+sys.path.insert(0, %r)
+from paper_2412_16187_b200 import HashEvictCache, device_error_count
+rng = np.random.default_rng(2024)
+out = []
+for trial in range(24):
+    B = int(rng.integers(1, 5)); H = int(rng.integers(1, 5)); G = int(rng.choice([1, 2, 3, 4, 5, 7, 8])); d = 128
+    b = int(rng.choice([4, 8, 13, 16, 24, 32, 33, 40, 64]))
+    cmax = int(rng.choice([130, 300, 700, 1500, 3000, 4096, 4500, 6000]))
+    budgets = rng.integers(max(40, cmax // 3), cmax + 1, size=B).astype(np.int32)
+    N = int(rng.integers(cmax // 2, 3 * cmax))
+    plens = rng.integers(0, N + 1, size=B).astype(np.int32); plens[0] = N
+    prot = rng.random() < 0.5
+    n_sink = int(rng.integers(0, 6)) if prot else 0
+    n_recent = int(rng.integers(0, 30)) if prot else 0
+    g = torch.Generator(device="cuda"); g.manual_seed(trial)
+    K = torch.randn(B, H, N, d, device="cuda", generator=g)
+    if rng.random() < 0.3:  # little variety in the keys: many equal distances
+        K = K[:, :, :1, :] + 0.05 * K
+    Q = torch.randn(B, H * G, N, d, device="cuda", generator=g)
+    K = K.to(torch.bfloat16); Q = Q.to(torch.bfloat16)
+    c = HashEvictCache(B, H, G, d, b, budgets, torch.randn(d, b, device="cuda", generator=g), dtype=torch.bfloat16,
+                       n_sink=n_sink, n_recent=n_recent)
+    c.prefill_compress(Q, K, K, torch.from_numpy(plens).cuda())
+    torch.cuda.synchronize()
+    h = hashlib.sha256()
+    for t in (c.codes, c.pos, c.scores, c.fill, c.next_pos):
+        h.update(t.cpu().numpy().tobytes())
+    out.append(h.hexdigest())
+assert device_error_count() == 0
+print("DIGESTS " + json.dumps(out))
+""" % (ROOT,)
+
+
+def test_replay_implementations_agree_on_random_shapes():
+    """Random group sizes (1..8), code widths (4..64, odd ones included), ragged budgets from 40 to 6000 slots, ragged
+    prompt lengths (empty and shorter than the budget included), protected windows, keys with little variety."""
+    def digests(env):
+        e = dict(os.environ, **env)
+        r = subprocess.run([sys.executable, "-c", RANDOM_SCRIPT], env=e, capture_output=True, text=True, timeout=900)
+        assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-4000:]
+        return json.loads([l for l in r.stdout.splitlines() if l.startswith("DIGESTS ")][-1][len("DIGESTS "):])
+
+    ref = digests({"HE_TC_REPLAY": "0"})
+    assert digests({"HE_TC_REPLAY": "1"}) == ref
+    assert digests({"HE_TC_REPLAY": "1", "HE_TC_REPLAY_BF16": "1"}) == ref
