@@ -311,7 +311,7 @@ int launch_replay_reg_one(const ReplayArgs& a, long long units, cudaStream_t str
     per_sm[dev] = n > 0 ? n : 1;
   }
   const int nbins = sms < kMaxBins ? sms : kMaxBins;
-  prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched);
+  prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched, 0);
   HE_CUDA_CHECK(cudaGetLastError());
   long long grid = (long long)sms * per_sm[dev];
   if (grid > units) grid = units;
@@ -345,7 +345,8 @@ int launch_replay_tc_one(const ReplayArgs& a0, long long units, cudaStream_t str
   int sms = 0;
   if (int rc = sm_count(&sms)) return rc;
   const int nbins = sms < kMaxBins ? sms : kMaxBins;
-  prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched);
+  // a step of this kernel costs about 400 cycles of resolver time plus 0.06 cycles per slot of tile work
+  prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched, 6700);
   HE_CUDA_CHECK(cudaGetLastError());
   const long long grid = units < sms ? units : sms;
   prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8, PROT><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);

@@ -19,7 +19,7 @@ struct ReplayArgs {
   const int32_t* prompt_len;
   long long Nmax;
   int smem_slots;  // slots the shared-memory tables were sized for
-  int32_t* sched;  // unit schedule written by prefill_schedule_kernel (register kernel only)
+  int32_t* sched;  // unit schedule written by prefill_schedule_kernel
 };
 
 constexpr int kStepBlock = 32;  // prompt tokens whose query contexts are staged at a time (one per lane of warp 0)
@@ -70,9 +70,11 @@ constexpr int kSchedThreads = 1024;
 
 __host__ __device__ inline size_t sched_words(long long units) { return 3 + 2 * (size_t)kMaxBins + (size_t)units; }
 
+// step_cost: fixed cost of one evicting step in units of one slot scanned (0 for the register kernel, whose step is a
+// scan; several thousand for the tensor-core kernel, whose step is mostly the resolver's latency).
 __global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const he_config cfg, const int32_t* budget,
                                                                           const int32_t* prompt_len, int nbins,
-                                                                          int32_t* sched) {
+                                                                          int32_t* sched, int step_cost) {
   __shared__ unsigned long long keys[kSchedSortMax];  // (work << 20) | (0xFFFFF - unit), sorted descending
   __shared__ int count[kMaxBins + 1];
   __shared__ unsigned char bin_of[kSchedSortMax];  // nbins <= 256
@@ -108,7 +110,7 @@ __global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const h
     if (i < units) {
       const int s = i / cfg.n_kv_heads;
       const long long C = budget[s], N = prompt_len[s];
-      const long long work = N > C ? (N - C) * C + 1 : 1;  // evicting steps x slots scanned
+      const long long work = N > C ? (N - C) * (C + step_cost) + 1 : 1;  // evicting steps x (slots scanned + fixed cost)
       key = ((unsigned long long)work << 20) | (unsigned long long)(0xFFFFF - i);
     }
     keys[i] = key;
