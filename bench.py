@@ -175,6 +175,9 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+PACKED_CODES = False  # set from --packed-codes
+
+
 def config_dict(w, replicas):
     return {
         "workload": w.name, "batch": w.batch, "layers_folded": w.layers, "n_kv_heads": w.n_kv_heads,
@@ -182,7 +185,7 @@ def config_dict(w, replicas):
         "budget": "ragged U[%d,%d]" % (w.budget_lo, w.budget_hi) if w.ragged else w.budget,
         "prompt_len": "%d x budget" % w.prompt_factor if w.ragged else w.prompt_len,
         "decode_steps": w.decode_steps, "layer_replicas": replicas, "n_sink": w.n_sink, "n_recent": w.n_recent,
-        "write_scores": True,
+        "write_scores": True, "packed_codes": bool(PACKED_CODES),
         "l2": "inputs larger than L2: every decode call streams a different layer replica's tables "
               "(replicas x per-call bytes > 126 MB); prefill reads GBs of prompt",
     }
@@ -227,7 +230,8 @@ def run_ours(args, w):
     gq, gk, gv = (up(wl.gen_decode_inputs(w, x, 0, T)) for x in "qkv")
     dplen = torch.from_numpy(plens).cuda()
     caches = [HashEvictCache(B, H, G, d, w.hash_bits, budgets, torch.from_numpy(wl.gen_W(w, layer=r)), dtype=tdt,
-                             n_sink=w.n_sink, n_recent=w.n_recent, write_scores=True) for r in range(R)]
+                             n_sink=w.n_sink, n_recent=w.n_recent, write_scores=True, packed_codes=args.packed_codes)
+              for r in range(R)]
     ws = caches[0].workspace(Nmax)
     victims = torch.empty((R, B, H), dtype=torch.int32, device="cuda")
     t_gen = time.perf_counter() - t_gen
@@ -348,10 +352,10 @@ def run_ours(args, w):
         # ---- secondary figure: the same decode kernel with all R replicas folded into ONE call (batch R*B), i.e. when
         # the per-call fixed costs (graph node, dependent load chain) are amortised over R times more units
         big = HashEvictCache(R * B, H, G, d, w.hash_bits, np.tile(budgets, R), torch.from_numpy(wl.gen_W(w)), dtype=tdt,
-                             n_sink=w.n_sink, n_recent=w.n_recent, write_scores=True)
+                             n_sink=w.n_sink, n_recent=w.n_recent, write_scores=True, packed_codes=args.packed_codes)
         for r, c in enumerate(caches):
             sl = slice(r * B, (r + 1) * B)
-            big.codes[sl].copy_(c.codes)
+            big.codes_storage[sl].copy_(c.codes_storage)
             big.pos[sl].copy_(c.pos)
             big.fill[sl].copy_(c.fill)
             big.next_pos[sl].copy_(c.next_pos)
@@ -477,6 +481,8 @@ def main():
     ap.add_argument("--replicas", type=int, default=None, help="independent layer replicas cycled by the decode loop")
     ap.add_argument("--decode-steps", type=int, default=None)
     ap.add_argument("--hash-bits", type=int, default=None, help="override b (hash-dimension sweep of Section 4.7)")
+    ap.add_argument("--packed-codes", action="store_true",
+                    help="code table with ceil(b/8) bytes per slot (HE_FLAG_PACKED_CODES) instead of 32-bit words")
     ap.add_argument("--batch", type=int, default=None, help="fewer sequences (profiling captures on a small case)")
     ap.add_argument("--prompt-factor", type=int, default=None, help="ragged workloads: prompt = factor x budget")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of a CUDA graph")
@@ -489,6 +495,8 @@ def main():
     ap.add_argument("--ref-seqs", type=int, default=12, help="sequences in the oracle's bounded sample")
     ap.add_argument("--ref-decode-steps", type=int, default=128)
     args = ap.parse_args()
+    global PACKED_CODES
+    PACKED_CODES = args.packed_codes
     w = wl.CONFIGS[args.workload]
     if args.decode_steps is not None:
         w = w.scaled(decode_steps=args.decode_steps)

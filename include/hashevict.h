@@ -22,6 +22,10 @@
  *   k_cache, v_cache  [B, Hkv, Cmax, d]   dtype of the config, rows 16-byte aligned
  *   codes             [B, Hkv, Cmax, Wd]  uint32; bit i of a code is the sign bit of column i of W,
  *                                         stored in word i/32 at bit i%32; unused high bits are 0
+ *                                         With HE_FLAG_PACKED_CODES: [B, Hkv, Cmax, ceil(b/8)] bytes instead, bit i in
+ *                                         byte i/8 at bit i%8 (1 byte per slot at b <= 8, as Section 4.7 prices it);
+ *                                         Cmax * ceil(b/8) must then be a multiple of 16. For b = 32 and b = 64 the
+ *                                         two layouts are the same bytes.
  *   scores            [B, Hkv, Cmax]      fp32, -(Hamming distance summed over the group)
  *   pos               [B, Hkv, Cmax]      int32 token position held by the slot, -1 = empty
  *   budget            [B]                 int32 C_s <= Cmax, read-only
@@ -50,6 +54,7 @@ enum { HE_DTYPE_F32 = 0, HE_DTYPE_BF16 = 1 };
 
 /* flags */
 #define HE_FLAG_WRITE_SCORES 1u /* store the per-slot scores of Eq. 5 on every evicting step */
+#define HE_FLAG_PACKED_CODES 2u /* he_cache.codes holds ceil(b/8) bytes per slot instead of Wd 32-bit words */
 
 typedef struct he_config {
   int32_t batch;      /* B; independent layers may be folded in by the caller */

@@ -15,6 +15,7 @@ from . import build as _build
 HE_OK = 0
 HE_DTYPE_F32, HE_DTYPE_BF16 = 0, 1
 HE_FLAG_WRITE_SCORES = 1
+HE_FLAG_PACKED_CODES = 2
 _DTYPES = {torch.float32: HE_DTYPE_F32, torch.bfloat16: HE_DTYPE_BF16}
 
 
@@ -137,19 +138,27 @@ class HashEvictCache:
     """Device-side cache state (the arrays of he_cache, allocated with torch) plus the calls that act on it."""
 
     def __init__(self, batch, n_kv_heads, group_size, head_dim, hash_bits, budgets, W, dtype=torch.bfloat16,
-                 max_budget=None, n_sink=0, n_recent=0, write_scores=True, device="cuda", host_budget_mirror=True):
+                 max_budget=None, n_sink=0, n_recent=0, write_scores=True, device="cuda", host_budget_mirror=True,
+                 packed_codes=False):
         lib()
         dev = torch.device(device)
         budgets = torch.as_tensor(budgets, dtype=torch.int32).reshape(-1)
         assert budgets.numel() == batch
         cmax = int(budgets.max()) if max_budget is None else int(max_budget)
         cmax = (cmax + 3) // 4 * 4  # the slot stride must keep 16-byte alignment
+        if packed_codes:
+            cmax = (cmax + 15) // 16 * 16  # ... also with one byte per slot
         self.B, self.H, self.G, self.d, self.b, self.Cmax = batch, n_kv_heads, group_size, head_dim, hash_bits, cmax
         self.Wd = (hash_bits + 31) // 32
         self.dtype = dtype
         self.k_cache = torch.zeros((batch, n_kv_heads, cmax, head_dim), dtype=dtype, device=dev)
         self.v_cache = torch.zeros_like(self.k_cache)
-        self.codes = torch.zeros((batch, n_kv_heads, cmax, self.Wd), dtype=torch.int32, device=dev)
+        # code table: Wd 32-bit words per slot, or ceil(b/8) bytes per slot with HE_FLAG_PACKED_CODES
+        self.packed_codes = bool(packed_codes)
+        if self.packed_codes:
+            self.codes_storage = torch.zeros((batch, n_kv_heads, cmax, (hash_bits + 7) // 8), dtype=torch.uint8, device=dev)
+        else:
+            self.codes_storage = torch.zeros((batch, n_kv_heads, cmax, self.Wd), dtype=torch.int32, device=dev)
         self.scores = torch.zeros((batch, n_kv_heads, cmax), dtype=torch.float32, device=dev)
         self.pos = torch.full((batch, n_kv_heads, cmax), -1, dtype=torch.int32, device=dev)
         self.budget = budgets.to(dev)
@@ -158,15 +167,25 @@ class HashEvictCache:
         self.W = W.to(device=dev, dtype=torch.float32).contiguous()
         assert self.W.shape == (head_dim, hash_bits)
         self.cfg = _config(batch, n_kv_heads, group_size, head_dim, hash_bits, cmax, n_sink, n_recent, dtype,
-                           HE_FLAG_WRITE_SCORES if write_scores else 0)
+                           (HE_FLAG_WRITE_SCORES if write_scores else 0) | (HE_FLAG_PACKED_CODES if packed_codes else 0))
         self._budget_host = (ctypes.c_int32 * batch)(*[int(x) for x in budgets.tolist()])  # host mirror of `budget`
-        self.ca = he_cache(*[_ptr(t) for t in (self.k_cache, self.v_cache, self.codes, self.scores, self.pos,
+        self.ca = he_cache(*[_ptr(t) for t in (self.k_cache, self.v_cache, self.codes_storage, self.scores, self.pos,
                                                self.budget, self.fill, self.next_pos, self.W)],
                            ctypes.cast(self._budget_host, ctypes.c_void_p) if host_budget_mirror else None, None)
         # scratch for the bulk-hashed decode step that large batches use (codes of the step's new rows)
         self.step_scratch = torch.empty(lib().he_step_scratch_bytes(ctypes.byref(self.cfg)), dtype=torch.uint8, device=dev)
         self.ca.step_scratch = _ptr(self.step_scratch)
         self._ws = None
+
+    @property
+    def codes(self):
+        """The code table as int32 words [B, Hkv, Cmax, Wd]: the storage itself, or (packed layout) a copy widened to words."""
+        if not self.packed_codes:
+            return self.codes_storage
+        raw = self.codes_storage
+        wide = torch.zeros(raw.shape[:-1] + (4 * self.Wd,), dtype=torch.uint8, device=raw.device)
+        wide[..., :raw.shape[-1]] = raw
+        return wide.view(torch.int32)
 
     # --- the four calls of the boundary -------------------------------------------------------------
     def reset(self, stream=None):

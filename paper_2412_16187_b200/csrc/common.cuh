@@ -18,6 +18,30 @@ constexpr uint32_t kKeyIdxMask = (1u << kKeyIdxBits) - 1u;
 __host__ __device__ inline int words_of(int b) { return (b + 31) >> 5; }
 __host__ __device__ inline int esize_of(int dtype) { return dtype == HE_DTYPE_BF16 ? 2 : 4; }
 
+// Bytes per slot of he_cache.codes in the packed layout (HE_FLAG_PACKED_CODES); 0 in the word layout, also where the
+// two layouts are the same bytes (25..32 and 57..64 bits).
+__host__ __device__ inline int packed_code_bytes(const he_config& cfg) {
+  const int cb = (cfg.flags & HE_FLAG_PACKED_CODES) ? (cfg.hash_bits + 7) >> 3 : 0;
+  return cb == 4 * words_of(cfg.hash_bits) ? 0 : cb;
+}
+
+// The code of one cache slot goes to he_cache.codes in the layout the config asks for. `code` holds WORDS words
+// (constant indices only, so it may live in registers).
+template <int WORDS>
+__device__ __forceinline__ void store_slot_code(const he_config& cfg, uint32_t* codes, long long slot_idx,
+                                                const uint32_t (&code)[WORDS]) {
+  const int cb = packed_code_bytes(cfg);
+  if (cb == 0) {
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w) codes[slot_idx * WORDS + w] = code[w];
+  } else {
+    uint8_t* dst = reinterpret_cast<uint8_t*>(codes) + slot_idx * cb;
+#pragma unroll
+    for (int i = 0; i < 4 * WORDS; ++i)
+      if (i < cb) dst[i] = (uint8_t)(code[i >> 2] >> (8 * (i & 3)));
+  }
+}
+
 __device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
 
 __device__ __forceinline__ uint32_t word_mask(int b, int w) {

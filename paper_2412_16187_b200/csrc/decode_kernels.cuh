@@ -42,8 +42,13 @@ __device__ __forceinline__ float neg_small_int(int D) { return 8388608.0f - __ui
 // kernels launched just before this one in the stream, which themselves started only after everything earlier had
 // finished. So the cache state and the step's k / v rows may be read BEFORE griddepcontrol.wait here; only new_codes
 // is read after it.
-template <int WORDS, int GT, int NT, bool PRE>
+//
+// PACKED = true (HE_FLAG_PACKED_CODES with fewer bytes per slot than the word layout; WORDS = 1): the table holds
+// cb = ceil(b/8) bytes per slot, 1 to 3. A thread takes four consecutive slots (cb words) at a time, widens each code
+// to a word in registers and scores it like a word-layout slot.
+template <int WORDS, int GT, int NT, bool PRE, bool PACKED = false>
 __global__ void __launch_bounds__(NT, (NT <= 256 ? (PRE ? 6 : 4) : 1)) decode_step_kernel(const DecodeArgs a) {
+  static_assert(!PACKED || WORDS == 1, "packed tables hold codes of at most 24 bits");
   constexpr int SPV = 4 / WORDS;  // slots per 16-byte vector
   constexpr int BP = 32 * WORDS;
   constexpr bool kGroupedCopy = WORDS == 2;
@@ -109,9 +114,11 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? (PRE ? 6 : 4) : 1)) decode_st
 
   // (1) code words -> shared memory, asynchronously. The copy is sized by the budget alone: if the unit turns out
   // to be still filling (fill < C) the copied words are simply not used.
-  const int nvec = (C * WORDS + 3) / 4;
+  const int cb = PACKED ? (b + 7) >> 3 : 0;
+  const int nvec = PACKED ? (C * cb + 15) / 16 : (C * WORDS + 3) / 4;
   {
-    const uint4* cvec = reinterpret_cast<const uint4*>(a.ca.codes + (size_t)unit * Cmax * WORDS);
+    const uint4* cvec = PACKED ? reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(a.ca.codes) + (size_t)unit * Cmax * cb)
+                               : reinterpret_cast<const uint4*>(a.ca.codes + (size_t)unit * Cmax * WORDS);
     // Two-word codes (b > 32): one commit group per vector of this thread; the scan waits for them one by one and
     // reads only what this thread copied itself, so it overlaps the rest of the transfer. Measured on B200 this is
     // 6 % faster per call at b = 64 but slower at b <= 32 (larger unrolled scan body), where a single group is used.
@@ -297,7 +304,63 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? (PRE ? 6 : 4) : 1)) decode_st
     };
     using T = std::true_type;
     using F = std::false_type;
-    if (prot) {
+    // packed table: CB bytes per slot; like a word-layout vector, a group is four consecutive slots (CB words)
+    auto scan_packed = [&](auto cb_c, auto prot_c, auto scores_c) {
+      constexpr int CB = decltype(cb_c)::value;
+      constexpr bool PROT = decltype(prot_c)::value, SCORES = decltype(scores_c)::value;
+      const int ngroups = (C + 3) / 4;
+#pragma unroll 2
+      for (int gi = tid; gi < ngroups; gi += NT) {
+        uint32_t wd[CB];
+        if (CB == 2) {
+          const uint2 x = *reinterpret_cast<const uint2*>(dsm + gi * CB);
+          wd[0] = x.x, wd[CB - 1] = x.y;
+        } else {
+#pragma unroll
+          for (int i = 0; i < CB; ++i) wd[i] = dsm[gi * CB + i];
+        }
+        const int j0 = gi * 4;
+        const bool whole = j0 + 4 <= C;
+        int rk[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          constexpr int kBits = 8 * CB;
+          const int o = e * kBits;  // bit offset of the slot's code inside the group
+          uint32_t h[WORDS] = {};  // WORDS is 1 wherever this runs
+          if (CB == 3) h[0] = __funnelshift_r(wd[o >> 5], wd[(o >> 5) + 1 < CB ? (o >> 5) + 1 : CB - 1], o & 31) & 0xFFFFFFu;
+          else h[0] = (wd[o >> 5] >> (o & 31)) & ((1u << kBits) - 1u);
+          rk[e] = ctx.rank(h);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j = j0 + e;
+          if (whole || j < C) {
+            const uint32_t key = ((uint32_t)rk[e] << kKeyIdxBits) + (kKeyBase - (uint32_t)j);
+            best_all = max(best_all, key);
+            if (PROT) {
+              const int p = __ldg(pp + j);
+              if (p >= cfg.n_sink && p < t - cfg.n_recent) best_el = max(best_el, key);
+            }
+            if (SCORES && !whole) sc[j] = neg_small_int(ctx.dist(rk[e]));
+          }
+        }
+        if (SCORES && whole)
+          *reinterpret_cast<float4*>(sc + j0) = make_float4(neg_small_int(ctx.dist(rk[0])), neg_small_int(ctx.dist(rk[1])),
+                                                            neg_small_int(ctx.dist(rk[2])), neg_small_int(ctx.dist(rk[3])));
+      }
+    };
+    auto scan_packed_cb = [&](auto prot_c, auto scores_c) {
+      if (cb == 1) scan_packed(std::integral_constant<int, 1>{}, prot_c, scores_c);
+      else if (cb == 2) scan_packed(std::integral_constant<int, 2>{}, prot_c, scores_c);
+      else scan_packed(std::integral_constant<int, 3>{}, prot_c, scores_c);
+    };
+    if constexpr (PACKED) {
+      if (prot) {
+        if (write_scores) scan_packed_cb(T{}, T{}); else scan_packed_cb(T{}, F{});
+      } else {
+        if (write_scores) scan_packed_cb(F{}, T{}); else scan_packed_cb(F{}, F{});
+      }
+    } else if (prot) {
       if (write_scores) scan(T{}, T{}); else scan(T{}, F{});
     } else {
       if (write_scores) scan(F{}, T{}); else scan(F{}, F{});
@@ -322,8 +385,12 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? (PRE ? 6 : 4) : 1)) decode_st
     int ev = -1;
     if (evict && a.evicted_pos_out != nullptr) ev = a.ca.pos[slot_idx];
     a.ca.pos[slot_idx] = t;
+    if (PACKED) {
+      for (int i = 0; i < cb; ++i) reinterpret_cast<uint8_t*>(a.ca.codes)[slot_idx * cb + i] = (uint8_t)(codes_s[G] >> (8 * i));
+    } else {
 #pragma unroll
-    for (int w = 0; w < WORDS; ++w) a.ca.codes[slot_idx * WORDS + w] = codes_s[G * WORDS + w];
+      for (int w = 0; w < WORDS; ++w) a.ca.codes[slot_idx * WORDS + w] = codes_s[G * WORDS + w];
+    }
     if (!evict) {
       a.ca.scores[slot_idx] = 0.f;
       a.ca.fill[unit] = fill + 1;

@@ -56,7 +56,12 @@ __global__ void reset_kernel(const he_config cfg, const he_cache ca) {
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < slots; i += stride) {
     ca.pos[i] = -1;
     ca.scores[i] = 0.f;
-    for (int w = 0; w < Wd; ++w) ca.codes[i * Wd + w] = 0u;
+    const int cb = packed_code_bytes(cfg);
+    if (cb == 0) {
+      for (int w = 0; w < Wd; ++w) ca.codes[i * Wd + w] = 0u;
+    } else {
+      for (int w = 0; w < cb; ++w) reinterpret_cast<uint8_t*>(ca.codes)[i * cb + w] = 0;
+    }
     if (i < units) {
       ca.fill[i] = 0;
       ca.next_pos[i] = 0;
@@ -79,6 +84,11 @@ int check_config(const he_config* cfg, bool need_cache_dims) {
   if (cfg->max_budget < 4 || cfg->max_budget % 4 != 0) return fail(HE_ERR_INVALID_ARG, "max_budget %d is not a positive multiple of 4", cfg->max_budget);
   if (cfg->max_budget > (1 << kKeyIdxBits)) return fail(HE_ERR_UNSUPPORTED, "max_budget %d > 2^20", cfg->max_budget);
   if (cfg->n_sink < 0 || cfg->n_recent < 0) return fail(HE_ERR_INVALID_ARG, "n_sink / n_recent must be >= 0");
+  if (const int cb = packed_code_bytes(*cfg)) {
+    if (cb > 3) return fail(HE_ERR_UNSUPPORTED, "packed codes of %d bytes per slot (hash_bits %d): 1 to 3, or whole words", cb, cfg->hash_bits);
+    if (((long long)cfg->max_budget * cb) % 16 != 0)
+      return fail(HE_ERR_INVALID_ARG, "packed codes: max_budget %d x %d bytes must be a multiple of 16", cfg->max_budget, cb);
+  }
   return HE_OK;
 }
 
@@ -245,9 +255,9 @@ int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments
   return HE_OK;
 }
 
-template <int WORDS, int GT, int NT, bool PRE>
+template <int WORDS, int GT, int NT, bool PRE, bool PACKED = false>
 int launch_decode_one(const DecodeArgs& a, size_t smem, dim3 grid, cudaStream_t stream) {
-  if (int rc = set_smem(decode_step_kernel<WORDS, GT, NT, PRE>, smem)) return rc;
+  if (int rc = set_smem(decode_step_kernel<WORDS, GT, NT, PRE, PACKED>, smem)) return rc;
   cudaLaunchConfig_t lc{};
   lc.gridDim = grid;
   lc.blockDim = dim3(NT);
@@ -258,28 +268,28 @@ int launch_decode_one(const DecodeArgs& a, size_t smem, dim3 grid, cudaStream_t 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
   lc.numAttrs = pdl_enabled() ? 1 : 0;
-  HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, decode_step_kernel<WORDS, GT, NT, PRE>, a));
+  HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, decode_step_kernel<WORDS, GT, NT, PRE, PACKED>, a));
   return HE_OK;
 }
 
-template <int WORDS, int GT>
+template <int WORDS, int GT, bool PACKED>
 int launch_decode_nt(const DecodeArgs& a, int nt, size_t smem, dim3 grid, cudaStream_t stream) {
   if (a.new_codes != nullptr) {
-    if (nt == 256) return launch_decode_one<WORDS, GT, 256, true>(a, smem, grid, stream);
-    if (nt == 512) return launch_decode_one<WORDS, GT, 512, true>(a, smem, grid, stream);
-    return launch_decode_one<WORDS, GT, 1024, true>(a, smem, grid, stream);
+    if (nt == 256) return launch_decode_one<WORDS, GT, 256, true, PACKED>(a, smem, grid, stream);
+    if (nt == 512) return launch_decode_one<WORDS, GT, 512, true, PACKED>(a, smem, grid, stream);
+    return launch_decode_one<WORDS, GT, 1024, true, PACKED>(a, smem, grid, stream);
   }
-  if (nt == 256) return launch_decode_one<WORDS, GT, 256, false>(a, smem, grid, stream);
-  if (nt == 512) return launch_decode_one<WORDS, GT, 512, false>(a, smem, grid, stream);
-  return launch_decode_one<WORDS, GT, 1024, false>(a, smem, grid, stream);
+  if (nt == 256) return launch_decode_one<WORDS, GT, 256, false, PACKED>(a, smem, grid, stream);
+  if (nt == 512) return launch_decode_one<WORDS, GT, 512, false, PACKED>(a, smem, grid, stream);
+  return launch_decode_one<WORDS, GT, 1024, false, PACKED>(a, smem, grid, stream);
 }
 
-template <int WORDS>
+template <int WORDS, bool PACKED = false>
 int launch_decode_g(const DecodeArgs& a, int nt, size_t smem, dim3 grid, cudaStream_t stream) {
   switch (a.cfg.group_size) {
-    case 1: return launch_decode_nt<WORDS, 1>(a, nt, smem, grid, stream);
-    case 4: return launch_decode_nt<WORDS, 4>(a, nt, smem, grid, stream);
-    default: return launch_decode_nt<WORDS, 0>(a, nt, smem, grid, stream);
+    case 1: return launch_decode_nt<WORDS, 1, PACKED>(a, nt, smem, grid, stream);
+    case 4: return launch_decode_nt<WORDS, 4, PACKED>(a, nt, smem, grid, stream);
+    default: return launch_decode_nt<WORDS, 0, PACKED>(a, nt, smem, grid, stream);
   }
 }
 
@@ -383,6 +393,8 @@ int launch_replay(const ReplayArgs& a, long long units, cudaStream_t stream) {
   if (int rc = sm_count(&sms)) return rc;
   const int min_budget = units <= sms ? 512 : 1152;
   bool tc_ok = mode != 0 && a.cfg.max_budget <= kRtMaxSlotsGlobal && (mode == 2 || a.cfg.max_budget >= min_budget);
+  // beyond 4096 slots the tensor-core kernel keeps its working table in the cache's own code array: word layout only
+  if (a.cfg.max_budget > kRtMaxSlots && packed_code_bytes(a.cfg) != 0) tc_ok = false;
   if (tc_ok && (a.cfg.n_sink > 0 || a.cfg.n_recent > 0)) {
     // protected windows: every budget must leave an eligible slot at every step (n_sink + n_recent < C), which the host
     // can only check on the caller's mirror of the budgets; with the tables in global memory the kernel tracks the
@@ -447,13 +459,15 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
   if (!q || !k || !v || !victim_out) return fail(HE_ERR_INVALID_ARG, "q, k, v or victim_out is null");
   if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return fail(HE_ERR_INVALID_ARG, "q, k, v must be 16-byte aligned");
   const int Wd = words_of(cfg->hash_bits);
-  const long long nvec = ((long long)cfg->max_budget * Wd + 3) / 4;
+  const int cb = packed_code_bytes(*cfg);  // 1..3 bytes per slot, or 0: word layout
+  const long long nvec = cb ? ((long long)cfg->max_budget * cb + 15) / 16 : ((long long)cfg->max_budget * Wd + 3) / 4;
   const size_t smem = (size_t)nvec * 16;
   if (smem > 200 * 1024) return fail(HE_ERR_UNSUPPORTED, "max_budget %d with %d code words does not fit the decode kernel's shared memory", cfg->max_budget, Wd);
   int nt = 256;
   if (nvec > 2048) nt = 512;
   if (nvec > 4096) nt = 1024;
-  if (nvec > 1024LL * kVecsPerThread)
+  if (cb) nt = cfg->max_budget <= 4096 ? 256 : (cfg->max_budget <= 16384 ? 512 : 1024);
+  if (!cb && nvec > 1024LL * kVecsPerThread)
     return fail(HE_ERR_UNSUPPORTED, "max_budget %d with %d code words exceeds the decode kernel's %d vectors", cfg->max_budget, Wd,
                 1024 * kVecsPerThread);
   if (cfg->batch > 65535) return fail(HE_ERR_UNSUPPORTED, "batch %d > 65535 in one decode call", cfg->batch);
@@ -504,6 +518,7 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
     memcpy(a.budget_vals, cache->budget_host, sizeof(int32_t) * (size_t)cfg->batch);
   }
   const dim3 grid((unsigned)cfg->n_kv_heads, (unsigned)cfg->batch);
+  if (cb) return launch_decode_g<1, true>(a, nt, smem, grid, st);
   return Wd == 1 ? launch_decode_g<1>(a, nt, smem, grid, st) : launch_decode_g<2>(a, nt, smem, grid, st);
 }
 

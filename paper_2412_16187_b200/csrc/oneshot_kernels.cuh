@@ -219,8 +219,10 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
   for (int i = b0; i < b1; ++i) {
     if (keys[i] <= thresh) {
       const long long dst = unit * Cmax + slot;
+      uint32_t cw[WORDS];
 #pragma unroll
-      for (int w = 0; w < WORDS; ++w) a.ca.codes[dst * WORDS + w] = kc_u[(long long)i * WORDS + w];
+      for (int w = 0; w < WORDS; ++w) cw[w] = kc_u[(long long)i * WORDS + w];
+      store_slot_code<WORDS>(a.cfg, a.ca.codes, dst, cw);
       a.ca.pos[dst] = i;
       const int n = N - 1 - i;
       a.ca.scores[dst] = POLICY == 0 ? (n > 0 ? -((float)S[i] / (float)n) : 0.f) : -__int_as_float(S[i]);
@@ -228,8 +230,10 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
     }
   }
   for (int j = keep + tid; j < Cmax; j += kOneshotThreads) {  // everything beyond `fill` is reset
+    uint32_t cw[WORDS];
 #pragma unroll
-    for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = 0u;
+    for (int w = 0; w < WORDS; ++w) cw[w] = 0u;
+    store_slot_code<WORDS>(a.cfg, a.ca.codes, unit * Cmax + j, cw);
     a.ca.pos[unit * Cmax + j] = -1;
     a.ca.scores[unit * Cmax + j] = 0.f;
   }
@@ -313,7 +317,11 @@ __global__ void __launch_bounds__(kStepL2Threads) decode_step_l2_kernel(const St
     if (fill >= C) ev = a.ca.pos[dst];
     a.ca.pos[dst] = t;
     a.ca.scores[dst] = -s_norm;
-    for (int w = 0; w < Wd; ++w) a.ca.codes[dst * Wd + w] = 0u;
+    if (const int cb = packed_code_bytes(a.cfg)) {
+      for (int w = 0; w < cb; ++w) reinterpret_cast<uint8_t*>(a.ca.codes)[dst * cb + w] = 0;
+    } else {
+      for (int w = 0; w < Wd; ++w) a.ca.codes[dst * Wd + w] = 0u;
+    }
     if (fill < C) a.ca.fill[unit] = fill + 1;
     a.ca.next_pos[unit] = t + 1;
     a.victim_out[unit] = slot;

@@ -356,8 +356,10 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : (NT <= 512 ? 2 : 1))) pre
       const int j = r * NT + tid;
       if (j < Cmax) {
         const bool valid = j < fill0;
+        uint32_t cw[WORDS];
 #pragma unroll
-        for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = valid ? code[r][w] : 0u;
+        for (int w = 0; w < WORDS; ++w) cw[w] = valid ? code[r][w] : 0u;
+        store_slot_code<WORDS>(a.cfg, a.ca.codes, unit * Cmax + j, cw);
         a.ca.pos[unit * Cmax + j] = valid ? pos_s[j] : -1;
         if (!(valid && scored)) sc[j] = 0.f;
       }
@@ -464,8 +466,10 @@ __global__ void prefill_replay_smem_kernel(const ReplayArgs a) {
   const bool scored = write_scores && N > C;
   for (int j = tid; j < Cmax; j += NT) {
     const bool valid = j < fill0;
+    uint32_t cw[WORDS];
 #pragma unroll
-    for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = valid ? codes_s[j * WORDS + w] : 0u;
+    for (int w = 0; w < WORDS; ++w) cw[w] = valid ? codes_s[j * WORDS + w] : 0u;
+    store_slot_code<WORDS>(a.cfg, a.ca.codes, unit * Cmax + j, cw);
     a.ca.pos[unit * Cmax + j] = valid ? pos_s[j] : -1;
     if (!(valid && scored)) sc[j] = 0.f;
   }

@@ -679,8 +679,10 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     for (int j = tid; j < Cmax; j += NT) {
       const bool valid = j < fill0;
       if (!GLOBAL_TABLE) {
+        uint32_t cw[WORDS];
 #pragma unroll
-        for (int w = 0; w < WORDS; ++w) a.ca.codes[(unit * Cmax + j) * WORDS + w] = valid ? codes_t[j * WORDS + w] : 0u;
+        for (int w = 0; w < WORDS; ++w) cw[w] = valid ? codes_t[j * WORDS + w] : 0u;
+        store_slot_code<WORDS>(a.cfg, a.ca.codes, unit * Cmax + j, cw);
         a.ca.pos[unit * Cmax + j] = valid ? pos_t[j] : -1;
       }
       if (!(valid && scored)) sc[j] = 0.f;
