@@ -157,6 +157,11 @@ int he_reset(const he_config* cfg, const he_cache* cache, void* stream);
  * back and synchronise `stream` before returning.
  *   he_decode_step_host:  q/k/v are host pointers laid out as for he_decode_step; victim_host [B, Hkv]
  *     receives the slots written. staging: >= he_decode_staging_bytes(cfg) device bytes.
+ *   he_decode_step_host_enqueue: the same copies and kernels put on `stream` WITHOUT the final synchronise, so that a
+ *     caller can keep several streams busy (say, the caches of different layers on alternating streams, each with
+ *     its own staging, copies of one overlapping the kernel of the other). victim_host holds the result, and
+ *     q/k/v_host and staging may be reused, only once `stream` has been synchronised; the host buffers must be
+ *     pinned for the copies to be asynchronous.
  *   he_prefill_compress_host: q [B, Hkv*G, Nmax, d], k, v [B, Hkv, Nmax, d] contiguous host tensors,
  *     prompt_len_host [B]; fill_host [B, Hkv] receives the valid-slot counts. staging: >=
  *     he_prefill_staging_bytes(cfg, max_prompt_len) device bytes (includes the prompt-code workspace).
@@ -164,6 +169,8 @@ int he_reset(const he_config* cfg, const he_cache* cache, void* stream);
 size_t he_decode_staging_bytes(const he_config* cfg);
 int he_decode_step_host(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
                         const void* v_host, int32_t* victim_host, void* staging, size_t staging_bytes, void* stream);
+int he_decode_step_host_enqueue(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
+                                const void* v_host, int32_t* victim_host, void* staging, size_t staging_bytes, void* stream);
 size_t he_prefill_staging_bytes(const he_config* cfg, int32_t max_prompt_len);
 int he_prefill_compress_host(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
                              const void* v_host, const int32_t* prompt_len_host, int32_t max_prompt_len,

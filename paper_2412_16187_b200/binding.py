@@ -36,7 +36,7 @@ class he_cache(ctypes.Structure):
 
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
-    "he_decode_staging_bytes", "he_decode_step_host", "he_prefill_staging_bytes", "he_prefill_compress_host",
+    "he_decode_staging_bytes", "he_decode_step_host", "he_decode_step_host_enqueue", "he_prefill_staging_bytes", "he_prefill_compress_host",
     "he_prefill_compress_noalloc", "he_attend", "he_prefill_oneshot", "he_oneshot_workspace_bytes", "he_prefill_oneshot_l2", "he_attention_loss", "he_decode_step_l2", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
 )
 
@@ -64,6 +64,7 @@ def lib():
     L.he_decode_staging_bytes.argtypes = [cfgp]
     L.he_decode_staging_bytes.restype = sz
     L.he_decode_step_host.argtypes = [cfgp, cap, vp, vp, vp, vp, vp, sz, vp]
+    L.he_decode_step_host_enqueue.argtypes = [cfgp, cap, vp, vp, vp, vp, vp, sz, vp]
     L.he_prefill_staging_bytes.argtypes = [cfgp, i32]
     L.he_prefill_staging_bytes.restype = sz
     L.he_prefill_compress_host.argtypes = [cfgp, cap, vp, vp, vp, vp, i32, vp, vp, sz, vp]
@@ -82,7 +83,7 @@ def lib():
     L.he_device_error_count.restype = ctypes.c_int
     L.he_last_error.argtypes = []
     L.he_last_error.restype = ctypes.c_char_p
-    for name in ("he_hash_keys", "he_decode_step", "he_prefill_compress", "he_reset", "he_decode_step_host",
+    for name in ("he_hash_keys", "he_decode_step", "he_prefill_compress", "he_reset", "he_decode_step_host", "he_decode_step_host_enqueue",
                  "he_prefill_compress_host", "he_prefill_compress_noalloc"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
@@ -289,6 +290,11 @@ class HashEvictCache:
     def decode_step_host(self, q_host, k_host, v_host, victim_host, staging, stream=None):
         _check(lib().he_decode_step_host(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q_host), _ptr(k_host),
                                          _ptr(v_host), _ptr(victim_host), _ptr(staging), staging.numel(), _stream(stream)))
+
+    def decode_step_host_enqueue(self, q_host, k_host, v_host, victim_host, staging, stream=None):
+        """he_decode_step_host_enqueue: as decode_step_host but without the final synchronise (results after a stream sync)."""
+        _check(lib().he_decode_step_host_enqueue(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q_host), _ptr(k_host),
+                                                 _ptr(v_host), _ptr(victim_host), _ptr(staging), staging.numel(), _stream(stream)))
 
     def prefill_compress_host(self, q_host, k_host, v_host, prompt_len_host, max_prompt_len, fill_host, staging, stream=None):
         _check(lib().he_prefill_compress_host(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q_host), _ptr(k_host),

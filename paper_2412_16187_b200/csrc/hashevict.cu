@@ -804,6 +804,13 @@ size_t he_decode_staging_bytes(const he_config* cfg) {
 
 int he_decode_step_host(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
                         const void* v_host, int32_t* victim_host, void* staging, size_t staging_bytes, void* stream) {
+  if (int rc = he_decode_step_host_enqueue(cfg, cache, q_host, k_host, v_host, victim_host, staging, staging_bytes, stream)) return rc;
+  HE_CUDA_CHECK(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  return HE_OK;
+}
+
+int he_decode_step_host_enqueue(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
+                                const void* v_host, int32_t* victim_host, void* staging, size_t staging_bytes, void* stream) {
   if (int rc = check_config(cfg, true)) return rc;
   if (!q_host || !k_host || !v_host || !victim_host || !staging) return fail(HE_ERR_INVALID_ARG, "a host pointer or staging is null");
   if ((reinterpret_cast<uintptr_t>(staging) & 255u) != 0) return fail(HE_ERR_INVALID_ARG, "staging must be 256-byte aligned");
@@ -825,7 +832,6 @@ int he_decode_step_host(const he_config* cfg, const he_cache* cache, const void*
   HE_CUDA_CHECK(cudaMemcpyAsync(dv, v_host, units * row, cudaMemcpyHostToDevice, st));
   if (int rc = he_decode_step(cfg, cache, dq, dk, dv, dvictim, nullptr, nullptr, stream)) return rc;
   HE_CUDA_CHECK(cudaMemcpyAsync(victim_host, dvictim, units * 4, cudaMemcpyDeviceToHost, st));
-  HE_CUDA_CHECK(cudaStreamSynchronize(st));
   return HE_OK;
 }
 

@@ -146,6 +146,32 @@ def test_host_buffer_variants_match_device_calls():
     assert torch.equal(a.gpu.codes, b.gpu.codes) and torch.equal(a.gpu.k_cache, b.gpu.k_cache)
 
 
+def test_enqueued_host_steps_on_two_streams_match_device_calls():
+    """he_decode_step_host_enqueue: two caches on two streams, several steps in flight, one synchronise at the end."""
+    from paper_2412_16187_b200 import decode_staging_bytes
+    w = PARITY_CASES["protected_tiny"]
+    steps = 12
+    ref, x, y = Case(w), Case(w), Case(w)
+    for c in (ref, x, y):
+        c.gpu.prefill_compress(c.dQ, c.dK, c.dV, c.dplen)
+    dq, dk, dv = (wl.gen_decode_inputs(w, n, 0, steps) for n in "qkv")
+    want = [ref.gpu.decode_step(to_dev(dq[i], w), to_dev(dk[i], w), to_dev(dv[i], w)).cpu() for i in range(steps)]
+    hq, hk, hv = (torch.from_numpy(t).pin_memory() for t in (dq, dk, dv))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    stagings = [torch.empty(decode_staging_bytes(x.gpu.cfg), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    got = torch.empty((2, steps, w.n_seq, w.n_kv_heads), dtype=torch.int32).pin_memory()
+    torch.cuda.synchronize()
+    for i in range(steps):
+        for ci, c in enumerate((x, y)):
+            c.gpu.decode_step_host_enqueue(hq[i], hk[i], hv[i], got[ci, i], stagings[ci], stream=streams[ci])
+    torch.cuda.synchronize()
+    for ci, c in enumerate((x, y)):
+        for i in range(steps):
+            assert torch.equal(got[ci, i], want[i]), (ci, i)
+        for name in ("codes", "pos", "scores", "k_cache", "v_cache", "fill", "next_pos"):
+            assert torch.equal(getattr(ref.gpu, name), getattr(c.gpu, name)), name
+
+
 def _sampled_full_size_check(w, seqs, decode_steps):
     """Full-size workload on the device in the launch configuration the benchmark times; the oracle replays only
     the sampled sequences (all their KV heads) on the device's codes and must reproduce their final state."""
