@@ -169,13 +169,28 @@ struct TcTile {
   int c2, c3;  // tensor-map coordinates of the segment (head, sequence)
 };
 
+// Dense schedule (prompt modes, batch within kTcLenCache): s_pref[s] counts the non-empty tiles of the sequences before
+// s (all heads), so tile numbers below s_pref[nseq] name non-empty tiles only and a strided walk over them gives every
+// CTA the same number of real tiles whatever the prompt lengths. `hint` is the caller's sequence cursor: tile numbers
+// only grow, so the search is a short walk forward. With nseq_dense = 0 tiles are numbered (segment, tile in segment)
+// and the empty ones are skipped.
 template <int WORDS>
 __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long long tiles_per_seg, TcTile* o,
-                                        const int* s_len, const int* s_bud) {
+                                        const int* s_len, const int* s_bud, const unsigned* s_pref, int nseq_dense, int* hint) {
   // 64-bit division is emulated and every role calls this once per tile: keep it to 32 bits whenever the counts fit
   int seg;
   long long ti;
-  if (job.mode == 0) {
+  if (nseq_dense > 0) {
+    int sq = *hint;
+    const unsigned tt = (unsigned)t;
+    while (sq + 1 < nseq_dense && s_pref[sq + 1] <= tt) ++sq;
+    *hint = sq;
+    const unsigned rem = tt - s_pref[sq];
+    const unsigned nt = (s_pref[sq + 1] - s_pref[sq]) / (unsigned)job.heads;  // tiles per head of this sequence (> 0 here)
+    const unsigned hh = rem / nt;
+    seg = sq * job.heads + (int)hh;
+    ti = (long long)(rem - hh * nt);
+  } else if (job.mode == 0) {
     seg = 0;
     ti = t;
   } else if (t < 0x7FFFFFFFll && tiles_per_seg < 0x7FFFFFFFll) {
@@ -237,6 +252,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   __shared__ uint32_t tmem_base_s;
   __shared__ volatile int abort_flag;
   __shared__ int s_len[kTcLenCache], s_bud[kTcLenCache];
+  __shared__ unsigned s_pref[kTcLenCache + 1];  // dense schedule: non-empty tiles (all heads) of the sequences before s
+  __shared__ int s_nseq_dense;
 
   // Programmatic dependent launch (used by the large-batch decode step): a kernel launched behind this one may
   // start right away; this kernel in turn finishes only after the kernel before it has (see the end).
@@ -275,13 +292,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  const int nseq = job.mode != 0 ? (int)(total_tiles / tiles_per_seg) / job.heads : 0;
   if (job.mode != 0) {
-    const int nseq = (int)(total_tiles / tiles_per_seg) / job.heads;
     for (int i = threadIdx.x; i < nseq && i < kTcLenCache; i += kTcThreads) {
       s_len[i] = job.prompt_len[i];
       s_bud[i] = job.budget[i];
     }
   }
+  if (tid == 0) s_nseq_dense = 0;
   // W -> three bf16 terms, transposed to [bit][channel] (K-major), 128B-swizzled; columns beyond b are zero.
   // Either copied from an image that a one-block-per-slice kernel prepared once for this call, or built here.
   if (job.w_image != nullptr) {
@@ -292,18 +310,50 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
     for (int idx = tid; idx < d * N; idx += kTcThreads) w_image_element(job.W, d, b, N, idx, Bs);
   }
   fence_proxy_async();  // the generic-proxy writes above are read by the tensor core through the async proxy
+  if (job.mode != 0 && nseq <= kTcLenCache && total_tiles < 0x7FFFFFFFll) {
+    __syncthreads();  // the cached lengths are complete
+    if (warp == 0) {  // exclusive prefix over the sequences' tile counts, 32 at a time
+      unsigned run = 0;
+      for (int i0 = 0; i0 < nseq; i0 += 32) {
+        const int i = i0 + lane;
+        unsigned cnt = 0;
+        if (i < nseq) {
+          const long long Ni = s_len[i], Ci = s_bud[i];
+          const long long r0 = (job.mode == 1 || job.q_all) ? 0 : (Ci < Ni ? Ci : Ni);
+          long long nt = Ni > r0 ? (Ni - r0 + kTcRows - 1) / kTcRows : 0;
+          if (nt > tiles_per_seg) nt = tiles_per_seg;
+          cnt = (unsigned)nt * (unsigned)job.heads;
+        }
+        unsigned inc = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+          if (lane >= o) inc += v;
+        }
+        if (i < nseq) s_pref[i] = run + inc - cnt;
+        run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+      }
+      if (lane == 0) {
+        s_pref[nseq] = run;
+        s_nseq_dense = nseq;
+      }
+    }
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
+  const int nseq_dense = s_nseq_dense;
+  const long long n_sched = nseq_dense > 0 ? (long long)s_pref[nseq_dense] : total_tiles;  // tile numbers this grid walks
+  int cursor = 0;  // this thread's sequence cursor of the dense schedule
 
   if (warp == 4 && TMA) {
     // ------------------------------------------------------------------ producer (TMA, one thread)
     if (lane == 0) {
       int it = 0;
-      for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      for (long long t = blockIdx.x; t < n_sched; t += gridDim.x) {
         TcTile tl;
-        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud)) continue;
+        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor)) continue;
         const int s = it % kTcStages;
         if (!mbar_wait(empty_bar(s), ((it / kTcStages) & 1) ^ 1, &abort_flag)) break;
         mbar_arrive_expect_tx(full_bar(s), (uint32_t)a_stage_bytes);
@@ -323,9 +373,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
       mbar_arrive(full_bar(published % kTcStages));
       ++published;
     };
-    for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+    for (long long t = blockIdx.x; t < n_sched && ok; t += gridDim.x) {
       TcTile tl;
-      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud)) continue;
+      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor)) continue;
       const int s = it % kTcStages;
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / kTcStages) & 1) ^ 1, &abort_flag));  // warp-uniform
       if (!ok) break;
@@ -354,9 +404,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
                              ((uint32_t)(kAccCols >> 3) << 17) | ((uint32_t)(kTcRows >> 4) << 24);
       const uint64_t b_desc0 = umma_desc_k128(smem_u32(Bs));
       int it = 0;
-      for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      for (long long t = blockIdx.x; t < n_sched; t += gridDim.x) {
         TcTile tl;
-        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud)) continue;
+        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor)) continue;
         const int s = it % kTcStages, acc = it & 1;
         // the epilogue has drained this accumulator and the stage's rows have landed
         if (!mbar_wait2(tempty_bar(acc), ((it >> 1) & 1) ^ 1, full_bar(s), (it / kTcStages) & 1, &abort_flag)) break;
@@ -382,9 +432,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-3, one row per thread)
     int it = 0;
-    for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+    for (long long t = blockIdx.x; t < n_sched; t += gridDim.x) {
       TcTile tl;
-      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud)) continue;
+      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor)) continue;
       const int acc = it & 1;
       if (!__all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(acc), (it >> 1) & 1, &abort_flag))) break;  // warp-uniform
       tc_fence_after();

@@ -76,8 +76,9 @@ __global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const h
                                                                           const int32_t* prompt_len, int nbins,
                                                                           int32_t* sched, int step_cost) {
   __shared__ unsigned long long keys[kSchedSortMax];  // (work << 20) | (0xFFFFF - unit), sorted descending
-  __shared__ int count[kMaxBins + 1];
+  __shared__ int start_s[kMaxBins];
   __shared__ unsigned char bin_of[kSchedSortMax];  // nbins <= 256
+  __shared__ unsigned short pos_of[kSchedSortMax];  // place of the unit inside its bin
   const int tid = threadIdx.x;
   const int units = cfg.batch * cfg.n_kv_heads;
   int32_t* bin_start = sched + 2;
@@ -131,21 +132,23 @@ __global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const h
       }
       __syncthreads();
     }
-  for (int i = tid; i < nbins; i += kSchedThreads) count[i] = 0;
-  __syncthreads();
   if (tid < 32) {  // greedy: next-largest unit to the lightest bin (lowest index on ties)
     // Bin loads live in registers (lane l owns bins l, l + 32, ...), scaled to 23 bits so that (load << 8 | bin) fits
     // one word and the lightest bin is a single redux.sync. The scaling only affects balance, never correctness.
+    // The owner lane of the chosen bin also counts the bin's units, so a unit's place inside its bin is known at once.
     constexpr int kOwn = kMaxBins / 32;
     unsigned long long total = 0ull;
     for (int i = tid; i < units; i += 32) total += keys[i] >> 20;
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
     int shift = 0;
     while ((total >> shift) >= (1ull << 23)) ++shift;
-    uint32_t own[kOwn];
+    uint32_t own[kOwn], cnt[kOwn];
 #pragma unroll
-    for (int k = 0; k < kOwn; ++k) own[k] = 0u;
+    for (int k = 0; k < kOwn; ++k) own[k] = 0u, cnt[k] = 0u;
+    unsigned long long key_next = units > 0 ? keys[0] : 0ull;
     for (int i = 0; i < units; ++i) {
+      const uint32_t wk = (uint32_t)((key_next >> 20) >> shift);
+      if (i + 1 < units) key_next = keys[i + 1];
       uint32_t best = 0xFFFFFFFFu;
 #pragma unroll
       for (int k = 0; k < kOwn; ++k) {
@@ -154,30 +157,37 @@ __global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const h
       }
       best = __reduce_min_sync(0xFFFFFFFFu, best);
       const int bb = (int)(best & 0xFFu);
-      const uint32_t wk = (uint32_t)((keys[i] >> 20) >> shift);
 #pragma unroll
       for (int k = 0; k < kOwn; ++k)
-        if (bb == tid + 32 * k) own[k] += wk;
-      if (tid == 0) {
-        bin_of[i] = (unsigned char)bb;
-        count[bb] += 1;
-      }
+        if (bb == tid + 32 * k) {
+          own[k] += wk;
+          bin_of[i] = (unsigned char)bb;
+          pos_of[i] = (unsigned short)cnt[k];
+          cnt[k] += 1u;
+        }
     }
+    // bin_start: exclusive prefix of the bins' counts (bin = lane + 32 k: prefix over lanes for each k, then over k)
+    uint32_t before_k = 0u;
+#pragma unroll
+    for (int k = 0; k < kOwn; ++k) {
+      uint32_t inc = cnt[k];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (tid >= o) inc += v;
+      }
+      const int bb = tid + 32 * k;
+      if (bb < nbins) {
+        start_s[bb] = (int)(before_k + inc - cnt[k]);
+        bin_start[bb] = (int)(before_k + inc - cnt[k]);
+      }
+      before_k += __shfl_sync(0xFFFFFFFFu, inc, 31);
+    }
+    if (tid == 0) bin_start[nbins] = units;
   }
   __syncthreads();
-  if (tid == 0) {
-    int acc = 0;
-    for (int b = 0; b < nbins; ++b) {
-      bin_start[b] = acc;
-      acc += count[b];
-      count[b] = 0;
-    }
-    bin_start[nbins] = acc;
-    for (int i = 0; i < units; ++i) {  // sorted order, so each bin lists its largest unit first
-      const int b = bin_of[i];
-      order[bin_start[b] + count[b]++] = 0xFFFFF - (int)(keys[i] & 0xFFFFF);
-    }
-  }
+  // sorted order, so each bin lists its largest unit first
+  for (int i = tid; i < units; i += kSchedThreads) order[start_s[bin_of[i]] + pos_of[i]] = 0xFFFFF - (int)(keys[i] & 0xFFFFF);
 }
 
 // Next unit for this CTA: from the bin of the SM it runs on, else from the first other bin that still has work.
