@@ -138,6 +138,11 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   constexpr int ESZ = FP8 ? 1 : 2;           // bytes per operand element
   constexpr int XATOM = (KB * ESZ) / 128, XCHUNK = ((KB * ESZ) % 128) / 16;  // where the key columns start
   constexpr int NSTAGE = FP8 ? 4 : 2;        // operand stages = accumulators in tensor memory
+  // Tiles per hand-over: with four stages two consecutive tiles (one per expander group) travel together, so every
+  // role waits on its mbarriers once per 256 slots instead of once per 128 (a wait costs about as much as a quarter
+  // of a tile's work even when the barrier is already complete).
+  constexpr int TP = FP8 ? 2 : 1;
+  constexpr int NSYNC = NSTAGE / TP;         // hand-over slots: stage pair (or stage) + accumulator pair (or accumulator)
   constexpr int NT = kRtThreads;
   extern __shared__ unsigned char rt_smem_raw[];
   __shared__ __align__(8) unsigned long long bars[4 * NSTAGE];
@@ -178,7 +183,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   if (tid == 0) {
     abort_flag = 0;
     for (int s = 0; s < NSTAGE; ++s) {
-      mbar_init(full_bar(s), 128);
+      mbar_init(full_bar(s), 128 * TP);
       mbar_init(tfull_bar(s), 1);
       mbar_init(tempty_bar(s), 4);
     }
@@ -214,7 +219,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
                          ((uint32_t)(kRtRows >> 4) << 24);
   const uint32_t kconst_bits = __float_as_uint((float)(G * KB / 2) * 16384.f) >> 16;  // exact: G K / 2 <= 256
   const uint32_t cst_e4m3 = rt_e4m3_of_int(G * KB / 2);
-  int it = 0;  // operand tiles processed so far; every role counts the same sequence
+  int it = 0;  // hand-overs (groups of TP tiles) so far; every role counts the same sequence
 
   for (;;) {
     if (warp == 0) {
@@ -341,15 +346,38 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
       const uint32_t* kb_codes = kraw + cur * kRtRows * WORDS;
       // ---- tiles 0 .. nbase-1: base slots; tile nbase: the block's own keys
       const int ntile = nbase + 1;
+      const int nsync = (ntile + TP - 1) / TP;
       if (warp >= 4 && warp < kRtMmaWarp) {
         // owner table cleared (-1: the slot still holds its base token); read only by the resolver
         for (int i = tid - 128; i < a.smem_slots / 2; i += 256) reinterpret_cast<uint32_t*>(owner)[i] = 0xFFFFFFFFu;
         // two groups of four warps, one per operand stage: group g expands the tiles that go to stage g
         const int x = (tid - 128) & 127, grp = (tid - 128) >> 7;  // x: this thread's row of the tile
-        for (int i = 0; i < ntile; ++i) {
-          const int n = it + i, st = n % NSTAGE, ph = (n / NSTAGE) & 1;
-          if ((n & 1) != grp) continue;
-          if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(st), ph ^ 1, &abort_flag))) break;
+        // Tables in global memory: a group's next base tile (two tiles on) is requested before this tile's wait and
+        // expansion, so the L2 latency of the code words is off the group's critical path. The table does not change
+        // during a block's tile phase.
+        uint32_t hn[WORDS];
+        auto fetch_next = [&](int i2) {
+          const int j2 = i2 * kRtTile + x;
+#pragma unroll
+          for (int w = 0; w < WORDS; ++w) hn[w] = (i2 < nbase && j2 < C) ? table_word(j2 * WORDS + w) : 0u;
+        };
+        if (GLOBAL_TABLE) fetch_next(TP == 1 ? ((it & 1) == grp ? 0 : 1) : grp);
+        for (int p = 0; p < nsync; ++p) {
+          const int n = it + p, ss = n % NSYNC, ph = (n / NSYNC) & 1;
+          if (TP == 1 && (n & 1) != grp) continue;
+          const int i = TP == 1 ? p : p * TP + grp;  // this group's tile of the hand-over
+          uint32_t hc[WORDS];
+          if (GLOBAL_TABLE) {
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) hc[w] = hn[w];
+            fetch_next(i + 2);
+          }
+          if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(ss), ph ^ 1, &abort_flag))) break;
+          if (i >= ntile) {  // the block's last hand-over is half empty
+            mbar_arrive(full_bar(ss));
+            continue;
+          }
+          const int st = TP == 1 ? ss : ss * TP + grp;
           unsigned char* bt = Bs + st * ATOMS * kRtAtomBytes;
           uint32_t h[WORDS];
           bool valid;
@@ -359,7 +387,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             valid = j < C;
             idx = kRtIdxMask - j;
 #pragma unroll
-            for (int w = 0; w < WORDS; ++w) h[w] = valid ? table_word(j * WORDS + w) : 0u;
+            for (int w = 0; w < WORDS; ++w) h[w] = GLOBAL_TABLE ? hc[w] : (valid ? table_word(j * WORDS + w) : 0u);
           } else {  // the block's own keys: plain distances, no index term
             valid = x < rows;
             idx = 0;
@@ -401,39 +429,50 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           }
           *reinterpret_cast<uint4*>(brow + XATOM * kRtAtomBytes + (((XCHUNK + 1) << 4) ^ xs)) = zero;
           fence_proxy_async();
-          mbar_arrive(full_bar(st));
+          mbar_arrive(full_bar(ss));
         }
       } else if (warp == kRtMmaWarp) {
         if (lane == 0) {
           const uint64_t a_desc0 = umma_desc_k128(smem_u32(As));
-          for (int i = 0; i < ntile; ++i) {
-            const int n = it + i, st = n % NSTAGE, ph = (n / NSTAGE) & 1;
-            // the readers have drained this accumulator and the expanders have written this operand stage
-            if (!mbar_wait2(tempty_bar(st), ph ^ 1, full_bar(st), ph, &abort_flag)) break;
+          for (int p = 0; p < nsync; ++p) {
+            const int n = it + p, ss = n % NSYNC, ph = (n / NSYNC) & 1;
+            // the readers have drained these accumulators and the expanders have written these operand stages
+            if (!mbar_wait2(tempty_bar(ss), ph ^ 1, full_bar(ss), ph, &abort_flag)) break;
             tc_fence_after();
-            const uint64_t b_desc0 = umma_desc_k128(smem_u32(Bs + st * ATOMS * kRtAtomBytes));
-            const uint32_t d_tmem = tmem_base + (uint32_t)(st * kRtTile);
 #pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-              if (FP8) {  // 32 one-byte columns per instruction
-                tc_mma_f8(d_tmem, a_desc0 + (uint64_t)((ks * 32) >> 4), b_desc0 + (uint64_t)((ks * 32) >> 4), idesc, ks > 0);
-              } else {
-                const uint32_t off = (uint32_t)(((ks * 16) / 64) * kRtAtomBytes + ((ks * 16) % 64) * 2);
-                tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)(off >> 4), b_desc0 + (uint64_t)(off >> 4), idesc, ks > 0);
+            for (int hf = 0; hf < TP; ++hf) {
+              if (p * TP + hf >= ntile) break;
+              const int st = ss * TP + hf;
+              const uint64_t b_desc0 = umma_desc_k128(smem_u32(Bs + st * ATOMS * kRtAtomBytes));
+              const uint32_t d_tmem = tmem_base + (uint32_t)(st * kRtTile);
+#pragma unroll
+              for (int ks = 0; ks < KSTEPS; ++ks) {
+                if (FP8) {  // 32 one-byte columns per instruction
+                  tc_mma_f8(d_tmem, a_desc0 + (uint64_t)((ks * 32) >> 4), b_desc0 + (uint64_t)((ks * 32) >> 4), idesc, ks > 0);
+                } else {
+                  const uint32_t off = (uint32_t)(((ks * 16) / 64) * kRtAtomBytes + ((ks * 16) % 64) * 2);
+                  tc_mma_bf16(d_tmem, a_desc0 + (uint64_t)(off >> 4), b_desc0 + (uint64_t)(off >> 4), idesc, ks > 0);
+                }
               }
             }
-            // one commit serves both consumers: when these MMAs are done the accumulator is complete (readers) and the
-            // operand stage may be rewritten (expanders); stage and accumulator share the index, so they share the barrier
-            tc_commit(tfull_bar(st));
+            // one commit serves both consumers: when these MMAs are done the accumulators are complete (readers) and the
+            // operand stages may be rewritten (expanders); stages and accumulators share the index, so they share the barrier
+            tc_commit(tfull_bar(ss));
           }
         }
       } else {
         bool ok = true;
-        for (int i = 0; i < ntile && ok; ++i) {
-          const int n = it + i, st = n % NSTAGE, ph = (n / NSTAGE) & 1;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(st), ph, &abort_flag));
+        for (int p = 0; p < nsync && ok; ++p) {
+          const int n = it + p, ss = n % NSYNC, ph = (n / NSYNC) & 1;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(ss), ph, &abort_flag));
           if (!ok) break;
           tc_fence_after();
+#pragma unroll
+          for (int hf = 0; hf < TP; ++hf) {
+          const int i = p * TP + hf;
+          if (i >= ntile) break;
+          const bool last_of_handover = hf == TP - 1 || i + 1 >= ntile;  // the accumulators go back after their last read
+          const int st = ss * TP + hf;
           const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(st * kRtTile);
           if (i < nbase) {  // the tile's largest key for this step (keys are non-negative floats: compare the bits)
             uint32_t mx = 0u;
@@ -446,9 +485,11 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
 #pragma unroll
               for (int k = 0; k < 32; ++k) mx = max(mx, max(v0[k], v1[k]));
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(st));
+            if (last_of_handover) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(tempty_bar(ss));
+            }
             Mx[tid * mp + i] = __float2int_rn(__uint_as_float(mx));
           } else {  // distances of the block's keys: key / 2^14, kept as 16-bit integers
 #pragma unroll
@@ -465,9 +506,12 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
 #pragma unroll
               for (int k = 0; k < 4; ++k) dst[k] = make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(st));
+            if (last_of_handover) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(tempty_bar(ss));
+            }
+          }
           }
         }
         if (ok) {
@@ -476,7 +520,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           RB[tid] = rb;
         }
       }
-      it += ntile;
+      it += nsync;
       tc_fence_before();
       __syncthreads();
       tc_fence_after();
