@@ -29,9 +29,9 @@ struct OneshotArgs {
   long long* sums_out;       // optional [units, Nmax]: S_i for the caller
 };
 
-constexpr int kOneshotThreads = 256;
+constexpr int kOneshotThreads = 512;
 constexpr int kOneshotWarps = kOneshotThreads / 32;
-constexpr int kOneshotSub = 64;  // tokens staged per warp at a time
+constexpr int kOneshotSub = 32;  // tokens staged per warp at a time
 constexpr unsigned long long kOneshotRanked = 1ull << 57;  // set in the keys of tokens outside the protected windows
 
 // Squared L2 norm of every prompt key in the precision that decides the L2 ranking: fp32, channels in ascending order,
@@ -114,6 +114,7 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
       const int nt = min(kOneshotSub, hi - j0);
       for (int x = lane; x < nt * GW; x += 32) qb[x] = __ldg(qc_u + (long long)j0 * GW + x);
       __syncwarp();
+#pragma unroll 4
       for (int x = 0; x < nt * G; ++x) {
 #pragma unroll
         for (int w = 0; w < WORDS; ++w) cnt[w] += (qb[x * WORDS + w] >> lane) & 1u;
@@ -133,6 +134,7 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
       for (int x = lane; x < nt * GW; x += 32) qb[x] = __ldg(qc_u + (long long)j0 * GW + x);
       for (int x = lane; x < nt * WORDS; x += 32) kb[x] = __ldg(kc_u + (long long)j0 * WORDS + x);
       __syncwarp();
+#pragma unroll 2
       for (int t = nt - 1; t >= 0; --t) {
         const int i = j0 + t;
         const int m = (N - 1 - i) * G;
@@ -180,7 +182,7 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
       s_want = keep;
     }
     for (int shift = 56; shift >= 0; shift -= 8) {
-      hist[tid] = 0u;  // 256 threads, 256 bins
+      if (tid < 256) hist[tid] = 0u;
       __syncthreads();
       const unsigned long long prefix = s_prefix;
       for (int i = tid; i < N; i += kOneshotThreads) {
