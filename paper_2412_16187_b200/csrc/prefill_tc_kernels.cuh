@@ -107,6 +107,13 @@ __device__ __forceinline__ uint4 rt_expand8(uint32_t byte) {
   return v;
 }
 
+// Largest of three floats in one instruction (sm_100 has the three-input form).
+__device__ __forceinline__ float rt_fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 // Group distance of Eq. 5 straight from the packed words (used for the few slots the resolver looks at itself).
 template <int WORDS>
 __device__ __forceinline__ int rt_dist(const uint32_t* h, const uint32_t* q, int G) {
@@ -183,7 +190,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   if (tid == 0) {
     abort_flag = 0;
     for (int s = 0; s < NSTAGE; ++s) {
-      mbar_init(full_bar(s), 128 * TP);
+      mbar_init(full_bar(s), 4 * TP);  // one arrival per expander warp
       mbar_init(tfull_bar(s), 1);
       mbar_init(tempty_bar(s), 4);
     }
@@ -374,7 +381,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           }
           if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(ss), ph ^ 1, &abort_flag))) break;
           if (i >= ntile) {  // the block's last hand-over is half empty
-            mbar_arrive(full_bar(ss));
+            if (lane == 0) mbar_arrive(full_bar(ss));
             continue;
           }
           const int st = TP == 1 ? ss : ss * TP + grp;
@@ -428,8 +435,9 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             *reinterpret_cast<uint4*>(brow + XATOM * kRtAtomBytes + ((XCHUNK << 4) ^ xs)) = zero;
           }
           *reinterpret_cast<uint4*>(brow + XATOM * kRtAtomBytes + (((XCHUNK + 1) << 4) ^ xs)) = zero;
-          fence_proxy_async();
-          mbar_arrive(full_bar(ss));
+          fence_proxy_async();  // every writing thread orders its stores before the async proxy, then one arrival per warp
+          __syncwarp();
+          if (lane == 0) mbar_arrive(full_bar(ss));
         }
       } else if (warp == kRtMmaWarp) {
         if (lane == 0) {
@@ -475,22 +483,33 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           const int st = ss * TP + hf;
           const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(st * kRtTile);
           if (i < nbase) {  // the tile's largest key for this step (keys are non-negative floats: compare the bits)
-            uint32_t mx = 0u;
-#pragma unroll
-            for (int c = 0; c < 4; c += 2) {  // two loads in flight per wait
-              uint32_t v0[32], v1[32];
-              tc_ld32(taddr + c * 32, v0);
-              tc_ld32(taddr + c * 32 + 32, v1);
+            float mxf;
+            {  // three loads in flight, the fourth issued before the first three are reduced: one exposed load latency per
+               // tile. The keys are non-negative whole numbers in fp32, so the floating-point maximum (three inputs per
+               // instruction, full-rate pipe) orders them like the integer one (two inputs, half rate); four running
+               // maxima keep the reduction from being one chain of dependent instructions.
+              uint32_t v0[32], v1[32], v2[32];
+              float m4[4] = {0.f, 0.f, 0.f, 0.f};
+              tc_ld32(taddr, v0);
+              tc_ld32(taddr + 32, v1);
+              tc_ld32(taddr + 64, v2);
               tc_wait_ld();
 #pragma unroll
-              for (int k = 0; k < 32; ++k) mx = max(mx, max(v0[k], v1[k]));
+              for (int k = 0; k < 32; k += 2) m4[(k >> 1) & 3] = rt_fmax3(m4[(k >> 1) & 3], __uint_as_float(v0[k]), __uint_as_float(v0[k + 1]));
+              tc_ld32(taddr + 96, v0);
+#pragma unroll
+              for (int k = 0; k < 32; ++k) m4[k & 3] = rt_fmax3(m4[k & 3], __uint_as_float(v1[k]), __uint_as_float(v2[k]));
+              tc_wait_ld();
+#pragma unroll
+              for (int k = 0; k < 32; k += 2) m4[(k >> 1) & 3] = rt_fmax3(m4[(k >> 1) & 3], __uint_as_float(v0[k]), __uint_as_float(v0[k + 1]));
+              mxf = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
             }
             if (last_of_handover) {
               tc_fence_before();
               __syncwarp();
               if (lane == 0) mbar_arrive(tempty_bar(ss));
             }
-            Mx[tid * mp + i] = __float2int_rn(__uint_as_float(mx));
+            Mx[tid * mp + i] = __float2int_rn(mxf);
           } else {  // distances of the block's keys: key / 2^14, kept as 16-bit integers
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
