@@ -35,3 +35,21 @@ def test_host_side_validation_needs_no_gpu():
     ca = binding.he_cache()
     assert L.he_reset(ctypes.byref(odd), ctypes.byref(ca), None) == 1 and b"max_budget" in L.he_last_error()
     assert L.he_reset(ctypes.byref(cfg), ctypes.byref(ca), None) == 1 and b"null" in L.he_last_error()
+
+
+def test_flag_values_match_the_header_and_packed_layout_is_validated_on_the_host():
+    text = open(os.path.join(ROOT, "include", "hashevict.h")).read()
+    flags = {m.group(1): int(m.group(2)) for m in re.finditer(r"#define\s+(HE_FLAG_[A-Z_]+)\s+(\d+)u", text)}
+    assert flags == {"HE_FLAG_WRITE_SCORES": binding.HE_FLAG_WRITE_SCORES, "HE_FLAG_PACKED_CODES": binding.HE_FLAG_PACKED_CODES}
+    L = binding.lib()
+    packed = binding.HE_FLAG_PACKED_CODES
+    ca = binding.he_cache()
+    # 40-bit codes would need 5 bytes per slot: only 1 to 3 bytes, or whole words, are stored
+    wide = binding.he_config(1, 1, 1, 128, 40, 64, 0, 0, 1, packed)
+    assert L.he_reset(ctypes.byref(wide), ctypes.byref(ca), None) == 2 and b"packed codes" in L.he_last_error()
+    # one byte per slot: the slot stride must keep units 16-byte aligned
+    ragged = binding.he_config(1, 1, 1, 128, 8, 36, 0, 0, 1, packed)
+    assert L.he_reset(ctypes.byref(ragged), ctypes.byref(ca), None) == 1 and b"multiple of 16" in L.he_last_error()
+    # 32- and 64-bit codes are the same bytes in both layouts: the flag changes nothing, the null cache is what fails
+    same = binding.he_config(1, 1, 1, 128, 64, 36, 0, 0, 1, packed)
+    assert L.he_reset(ctypes.byref(same), ctypes.byref(ca), None) == 1 and b"null" in L.he_last_error()
