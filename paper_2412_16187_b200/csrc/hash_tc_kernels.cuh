@@ -405,8 +405,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
       const uint64_t b_desc0 = umma_desc_k128(smem_u32(Bs));
       int it = 0;
       for (long long t = blockIdx.x; t < n_sched; t += gridDim.x) {
-        TcTile tl;
-        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor)) continue;
+        // flat rows and the dense schedule number real tiles only; otherwise empty tiles are skipped like the other
+        // roles skip them (this thread needs nothing else of the tile, so it avoids the index arithmetic)
+        if (job.mode != 0 && nseq_dense == 0) {
+          TcTile tl;
+          if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor)) continue;
+        }
         const int s = it % kTcStages, acc = it & 1;
         // the epilogue has drained this accumulator and the stage's rows have landed
         if (!mbar_wait2(tempty_bar(acc), ((it >> 1) & 1) ^ 1, full_bar(s), (it / kTcStages) & 1, &abort_flag)) break;
