@@ -178,7 +178,7 @@ template <int WORDS>
 __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long long tiles_per_seg, TcTile* o,
                                         const int* s_len, const int* s_bud, const unsigned* s_pref, int nseq_dense, int* hint) {
   // 64-bit division is emulated and every role calls this once per tile: keep it to 32 bits whenever the counts fit
-  int seg;
+  int seg, s_d = 0, hh_d = 0;  // dense schedule: sequence and head are known without dividing again
   long long ti;
   if (nseq_dense > 0) {
     int sq = *hint;
@@ -188,7 +188,9 @@ __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long lo
     const unsigned rem = tt - s_pref[sq];
     const unsigned nt = (s_pref[sq + 1] - s_pref[sq]) / (unsigned)job.heads;  // tiles per head of this sequence (> 0 here)
     const unsigned hh = rem / nt;
-    seg = sq * job.heads + (int)hh;
+    seg = 0;
+    s_d = sq;
+    hh_d = (int)hh;
     ti = (long long)(rem - hh * nt);
   } else if (job.mode == 0) {
     seg = 0;
@@ -212,7 +214,7 @@ __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long lo
     o->c2 = 0;
     o->c3 = 0;
   } else {
-    const int s = seg / job.heads, hh = seg % job.heads;
+    const int s = nseq_dense > 0 ? s_d : seg / job.heads, hh = nseq_dense > 0 ? hh_d : seg % job.heads;
     // lengths come from the CTA's shared-memory copy when the batch fits it: skipping an empty tile is then cheap
     const long long N = s < kTcLenCache ? s_len[s] : job.prompt_len[s];
     const long long C = s < kTcLenCache ? s_bud[s] : job.budget[s];
