@@ -230,7 +230,8 @@ def run_ours(args, w):
     gq, gk, gv = (up(wl.gen_decode_inputs(w, x, 0, T)) for x in "qkv")
     dplen = torch.from_numpy(plens).cuda()
     caches = [HashEvictCache(B, H, G, d, w.hash_bits, budgets, torch.from_numpy(wl.gen_W(w, layer=r)), dtype=tdt,
-                             n_sink=w.n_sink, n_recent=w.n_recent, write_scores=True, packed_codes=args.packed_codes)
+                             n_sink=w.n_sink, n_recent=w.n_recent, write_scores=True, packed_codes=args.packed_codes,
+                             early_inputs=not args.no_early_inputs)
               for r in range(R)]
     ws = caches[0].workspace(Nmax)
     victims = torch.empty((R, B, H), dtype=torch.int32, device="cuda")
@@ -367,7 +368,8 @@ def run_ours(args, w):
         # ---- secondary figure: the same decode kernel with all R replicas folded into ONE call (batch R*B), i.e. when
         # the per-call fixed costs (graph node, dependent load chain) are amortised over R times more units
         big = HashEvictCache(R * B, H, G, d, w.hash_bits, np.tile(budgets, R), torch.from_numpy(wl.gen_W(w)), dtype=tdt,
-                             n_sink=w.n_sink, n_recent=w.n_recent, write_scores=True, packed_codes=args.packed_codes)
+                             n_sink=w.n_sink, n_recent=w.n_recent, write_scores=True, packed_codes=args.packed_codes,
+                             early_inputs=not args.no_early_inputs)
         for r, c in enumerate(caches):
             sl = slice(r * B, (r + 1) * B)
             big.codes_storage[sl].copy_(c.codes_storage)
@@ -501,6 +503,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="fewer sequences (profiling captures on a small case)")
     ap.add_argument("--prompt-factor", type=int, default=None, help="ragged workloads: prompt = factor x budget")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of a CUDA graph")
+    ap.add_argument("--no-early-inputs", action="store_true",
+                    help="leave HE_FLAG_EARLY_INPUTS off (q, k, v are then read only after the stream's previous kernel has ended)")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-oneshot", action="store_true", help="skip the he_prefill_oneshot figure")

@@ -55,6 +55,8 @@ enum { HE_DTYPE_F32 = 0, HE_DTYPE_BF16 = 1 };
 /* flags */
 #define HE_FLAG_WRITE_SCORES 1u /* store the per-slot scores of Eq. 5 on every evicting step */
 #define HE_FLAG_PACKED_CODES 2u /* he_cache.codes holds ceil(b/8) bytes per slot instead of Wd 32-bit words */
+#define HE_FLAG_EARLY_INPUTS 4u /* he_decode_step may read q, k, v before the stream's earlier work has finished:
+                                   see he_decode_step */
 
 typedef struct he_config {
   int32_t batch;      /* B; independent layers may be folded in by the caller */
@@ -112,7 +114,20 @@ int he_hash_keys(const he_config* cfg, const void* x, int64_t rows, int64_t row_
  * Then K, V, code and pos of that slot are overwritten by k, v, h(k), t; next_pos and fill advance.
  * victim_out [B, Hkv]: slot written. evicted_pos_out [B, Hkv] (nullable): position that was evicted,
  * -1 when appended. qcodes_out [B, Hkv*G, Wd] (nullable): the query codes that were used.
- * The scores array is written only with HE_FLAG_WRITE_SCORES.
+ * The scores array is written only with HE_FLAG_WRITE_SCORES. A sequence whose budget is < 1 holds nothing: its units
+ * are left untouched and report victim -1.
+ *
+ * Ordering against earlier work of the stream. The kernel is launched with the programmatic-serialization attribute,
+ * so it may start while the stream's previous kernel is still running. By default it reads only W (which must not
+ * change while the cache is in use) before it waits for that kernel to finish; q, k, v may therefore be produced by
+ * the kernel enqueued just before this call. With HE_FLAG_EARLY_INPUTS the call also reads q, k, v and hashes them
+ * (Eq. 2) BEFORE that wait, so that this work overlaps the previous call's scan: consecutive decode calls (say, the
+ * caches of a model's layers one after another, or one cache step after step) then run about twice as fast. The
+ * caller promises in exchange that q, k, v were completely written before this call was ENQUEUED on the stream's
+ * device timeline - by work the host has synchronised with, or by work ordered before everything still pending in
+ * the stream (inputs staged ahead of a run of calls, or a captured graph whose inputs are final before it is
+ * launched). If the rows are produced by a kernel enqueued shortly before the call, leave the flag off. Results are
+ * identical with and without the flag.
  */
 int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, const void* k, const void* v,
                    int32_t* victim_out, int32_t* evicted_pos_out, uint32_t* qcodes_out, void* stream);

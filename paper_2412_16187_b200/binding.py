@@ -16,6 +16,7 @@ HE_OK = 0
 HE_DTYPE_F32, HE_DTYPE_BF16 = 0, 1
 HE_FLAG_WRITE_SCORES = 1
 HE_FLAG_PACKED_CODES = 2
+HE_FLAG_EARLY_INPUTS = 4
 _DTYPES = {torch.float32: HE_DTYPE_F32, torch.bfloat16: HE_DTYPE_BF16}
 
 
@@ -140,7 +141,7 @@ class HashEvictCache:
 
     def __init__(self, batch, n_kv_heads, group_size, head_dim, hash_bits, budgets, W, dtype=torch.bfloat16,
                  max_budget=None, n_sink=0, n_recent=0, write_scores=True, device="cuda", host_budget_mirror=True,
-                 packed_codes=False):
+                 packed_codes=False, early_inputs=False):
         lib()
         dev = torch.device(device)
         budgets = torch.as_tensor(budgets, dtype=torch.int32).reshape(-1)
@@ -168,7 +169,8 @@ class HashEvictCache:
         self.W = W.to(device=dev, dtype=torch.float32).contiguous()
         assert self.W.shape == (head_dim, hash_bits)
         self.cfg = _config(batch, n_kv_heads, group_size, head_dim, hash_bits, cmax, n_sink, n_recent, dtype,
-                           (HE_FLAG_WRITE_SCORES if write_scores else 0) | (HE_FLAG_PACKED_CODES if packed_codes else 0))
+                           (HE_FLAG_WRITE_SCORES if write_scores else 0) | (HE_FLAG_PACKED_CODES if packed_codes else 0) |
+                           (HE_FLAG_EARLY_INPUTS if early_inputs else 0))
         self._budget_host = (ctypes.c_int32 * batch)(*[int(x) for x in budgets.tolist()])  # host mirror of `budget`
         self.ca = he_cache(*[_ptr(t) for t in (self.k_cache, self.v_cache, self.codes_storage, self.scores, self.pos,
                                                self.budget, self.fill, self.next_pos, self.W)],

@@ -247,6 +247,11 @@ __device__ __forceinline__ void cp_async_wait_pending(int pending) {
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;\n" ::: "memory"); }
 
+// Asks for `bytes` (a multiple of 16, from a 16-byte aligned address) to be brought into L2. A hint: no data returns.
+__device__ __forceinline__ void l2_prefetch_bulk(const void* gmem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(gmem), "r"(bytes) : "memory");
+}
+
 // Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may start while
 // the previous kernel of the stream is still draining. Everything that touches memory another kernel may have
 // written comes after griddep_wait(); only W (read-only while a cache is in use) is read before it.

@@ -28,7 +28,9 @@ struct DecodeArgs {
   uint32_t* qcodes_out;
   const uint32_t* new_codes;               // PRE kernels: [B*Hkv*G + B*Hkv, Wd] codes of this step's q rows, then k rows
   int n_budget_vals;                       // > 0: budgets are in budget_vals (copied from he_cache.budget_host)
+  int n_sched;                             // > 0: sched lists the sequences by budget, largest first (sequence << 21 | budget)
   int32_t budget_vals[kMaxBudgetVals];
+  uint32_t sched[kMaxBudgetVals];
 };
 
 constexpr int kVecsPerThread = 8;  // 16-byte code vectors per thread (the host picks the block size accordingly)

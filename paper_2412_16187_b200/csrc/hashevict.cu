@@ -10,6 +10,7 @@
 // from 0; the partial sums are added in ascending chunk order; the bit is (sum >= 0).
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
@@ -21,6 +22,7 @@
 #include "attend_kernels.cuh"
 #include "common.cuh"
 #include "decode_kernels.cuh"
+#include "decode_sm_kernels.cuh"
 #include "hash_kernels.cuh"
 #include "hash_tc_kernels.cuh"
 #include "hashevict.h"
@@ -132,6 +134,13 @@ bool pdl_enabled() {
   return on;
 }
 
+// Environment switches are read once per process (ID separates the call sites' caches).
+template <int ID>
+bool env_flag_set(const char* name) {
+  static const bool on = getenv(name) != nullptr;
+  return on;
+}
+
 bool tc_enabled() {
   static const bool on = [] {
     const char* e = getenv("HE_DISABLE_TC");
@@ -166,7 +175,7 @@ bool encode_rows_tmap(const HashJob& job, long long max_rows_per_segment, int se
     return reinterpret_cast<EncodeFn>(fn);
   }();
   memset(out, 0, sizeof(*out));
-  if (encode == nullptr || getenv("HE_DISABLE_TMA") != nullptr) return false;
+  if (encode == nullptr || env_flag_set<2>("HE_DISABLE_TMA")) return false;
   cuuint64_t dims[4], strides[3];
   dims[0] = (cuuint64_t)job.d;
   if (job.mode == 0) {
@@ -293,6 +302,67 @@ int launch_decode_g(const DecodeArgs& a, int nt, size_t smem, dim3 grid, cudaStr
   }
 }
 
+// One CTA per SM (decode_sm_kernels.cuh), for HE_FLAG_EARLY_INPUTS: q, k, v are read and hashed before the wait.
+template <int WORDS, int GT, bool MMA>
+int launch_decode_sm_one(const DecodeArgs& a, unsigned grid, cudaStream_t stream) {
+  const size_t smem = sm_layout(a.cfg.head_dim, WORDS, esize_of(a.cfg.dtype), MMA).total;
+  if (int rc = set_smem(decode_step_sm_kernel<WORDS, GT, MMA>, smem)) return rc;
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3(grid);
+  lc.blockDim = dim3(kSmThreads);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = pdl_enabled() ? 1 : 0;
+  HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, decode_step_sm_kernel<WORDS, GT, MMA>, a));
+  return HE_OK;
+}
+
+template <int WORDS, int GT>
+int launch_decode_sm_g(const DecodeArgs& a, bool mma, unsigned grid, cudaStream_t stream) {
+  return mma ? launch_decode_sm_one<WORDS, GT, true>(a, grid, stream) : launch_decode_sm_one<WORDS, GT, false>(a, grid, stream);
+}
+
+template <int WORDS>
+int launch_decode_sm(const DecodeArgs& a, bool mma, unsigned grid, cudaStream_t stream) {
+  switch (a.cfg.group_size) {
+    case 1: return launch_decode_sm_g<WORDS, 1>(a, mma, grid, stream);
+    case 4: return launch_decode_sm_g<WORDS, 4>(a, mma, grid, stream);
+    default: return launch_decode_sm_g<WORDS, 0>(a, mma, grid, stream);
+  }
+}
+
+// Sequences ordered by budget, largest first (ties by index), each with its budget, for the unit schedule of the
+// one-CTA-per-SM decode kernel: word = sequence << 21 | budget. The caller's budget mirror is hashed on every call
+// and sorted again only when its contents changed.
+struct SchedCache {
+  uint64_t hash = 0;
+  int n = -1;
+  int cmax = 0;
+  uint32_t sched[kMaxBudgetVals];
+};
+const uint32_t* sched_of(const int32_t* budget_host, int n, int cmax) {
+  thread_local SchedCache c;
+  uint64_t h = 1469598103934665603ull;
+  for (int i = 0; i < n; ++i) h = (h ^ (uint32_t)budget_host[i]) * 1099511628211ull;
+  if (c.n != n || c.hash != h || c.cmax != cmax) {
+    uint16_t order[kMaxBudgetVals];
+    for (int i = 0; i < n; ++i) order[i] = (uint16_t)i;
+    std::stable_sort(order, order + n, [&](uint16_t x, uint16_t y) { return budget_host[x] > budget_host[y]; });
+    for (int i = 0; i < n; ++i) {
+      const int cb = budget_host[order[i]];
+      c.sched[i] = ((uint32_t)order[i] << kSmSchedShift) | (uint32_t)(cb < 0 ? 0 : (cb > cmax ? cmax : cb));
+    }
+    c.n = n;
+    c.hash = h;
+    c.cmax = cmax;
+  }
+  return c.sched;
+}
+
 template <int WORDS, int GT>
 int launch_replay_smem(const ReplayArgs& a, long long units, cudaStream_t stream) {
   const size_t smem = (size_t)a.cfg.max_budget * (WORDS + 1) * 4;
@@ -367,8 +437,11 @@ int launch_replay_tc_one(const ReplayArgs& a0, long long units, cudaStream_t str
 // 8-bit operands when the group's code sum fits e5m2 exactly (group sizes up to 7); HE_TC_REPLAY_BF16=1 keeps bf16.
 template <int WORDS, bool GLOBAL_TABLE>
 int launch_replay_tc(const ReplayArgs& a, long long units, cudaStream_t stream) {
-  const char* e = getenv("HE_TC_REPLAY_BF16");
-  const bool fp8 = a.cfg.group_size <= 7 && !(e && e[0] == '1');
+  static const bool bf16_forced = [] {
+    const char* e = getenv("HE_TC_REPLAY_BF16");
+    return e && e[0] == '1';
+  }();
+  const bool fp8 = a.cfg.group_size <= 7 && !bf16_forced;
   if (a.cfg.n_sink > 0 || a.cfg.n_recent > 0)  // protected windows
     return fp8 ? launch_replay_tc_one<WORDS, GLOBAL_TABLE, true, true>(a, units, stream)
                : launch_replay_tc_one<WORDS, GLOBAL_TABLE, false, true>(a, units, stream);
@@ -381,9 +454,12 @@ int launch_replay_tc(const ReplayArgs& a, long long units, cudaStream_t stream) 
 // kernel several units per SM at a cost that grows with the budget; measured on B200 (512 units, b = 64, G = 4) they
 // cross between 1024 and 1280 slots, and with no more units than SMs already around 512 slots.
 int tc_replay_mode() {
-  const char* e = getenv("HE_TC_REPLAY");
-  if (!tc_enabled() || (e && e[0] == '0')) return 0;
-  return (e && e[0] == '1') ? 2 : 1;
+  static const int mode = [] {
+    const char* e = getenv("HE_TC_REPLAY");
+    if (!tc_enabled() || (e && e[0] == '0')) return 0;
+    return (e && e[0] == '1') ? 2 : 1;
+  }();
+  return mode;
 }
 
 template <int WORDS>
@@ -483,13 +559,30 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
   a.evicted_pos_out = evicted_pos_out;
   a.qcodes_out = qcodes_out;
   a.n_budget_vals = 0;
+  a.n_sched = 0;
   a.new_codes = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // Large batches: hash the step's new rows with the bulk projection kernels (tensor cores for bf16) into the
   // caller's scratch, so the per-unit kernel only scans. Small batches keep the single fused kernel.
   const long long units_ll = (long long)cfg->batch * cfg->n_kv_heads;
+  // HE_FLAG_EARLY_INPUTS: while the units fit four per SM-wide CTA, the one-CTA-per-SM kernel hashes the step's rows
+  // before its wait. It serves whole-chunk head sizes with the word layout of the code table; larger batches keep the
+  // per-unit kernels (many waves of small CTAs hide their own latencies).
+  int sms = 0;
+  if (int rc = sm_count(&sms)) return rc;
+  const bool early = cb == 0 && cfg->head_dim % kChunk == 0 && (cfg->flags & HE_FLAG_EARLY_INPUTS) != 0 &&
+                     units_ll <= (long long)kSmUnits * sms && !env_flag_set<0>("HE_DISABLE_EARLY_DECODE");
+  if (early) {
+    if (cache->budget_host != nullptr && cfg->batch <= kMaxBudgetVals) {
+      a.n_sched = cfg->batch;
+      memcpy(a.sched, sched_of(cache->budget_host, cfg->batch, cfg->max_budget), sizeof(uint32_t) * (size_t)cfg->batch);
+    }
+    const unsigned g = (unsigned)(units_ll < sms ? units_ll : sms);
+    const bool mma = tc_enabled() && cfg->dtype == HE_DTYPE_BF16 && cfg->head_dim <= 128;
+    return Wd == 1 ? launch_decode_sm<1>(a, mma, g, st) : launch_decode_sm<2>(a, mma, g, st);
+  }
   if (cache->step_scratch != nullptr && units_ll * (cfg->group_size + 1) >= kSplitDecodeRows &&
-      getenv("HE_DISABLE_SPLIT_DECODE") == nullptr) {
+      !env_flag_set<1>("HE_DISABLE_SPLIT_DECODE")) {
     HashJob job{};
     job.W = cache->W;
     job.mode = 0;

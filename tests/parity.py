@@ -46,7 +46,7 @@ def check_hash_stage(x_np: np.ndarray, W: np.ndarray, dtype: str, gpu_codes: np.
 class Case:
     """One workload resident on both sides."""
 
-    def __init__(self, w, write_scores=True, packed_codes=False):
+    def __init__(self, w, write_scores=True, packed_codes=False, early_inputs=False):
         self.w = w
         self.W = wl.gen_W(w)
         self.plen = w.prompt_lens()
@@ -56,7 +56,7 @@ class Case:
         self.V = wl.gen_tokens(w, "v", 0, w.n_seq, 0, Nmax)
         self.gpu = HashEvictCache(w.n_seq, w.n_kv_heads, w.group_size, w.head_dim, w.hash_bits, w.budgets(),
                                   torch.from_numpy(self.W), dtype=torch_dtype(w), n_sink=w.n_sink, n_recent=w.n_recent,
-                                  write_scores=write_scores, packed_codes=packed_codes)
+                                  write_scores=write_scores, packed_codes=packed_codes, early_inputs=early_inputs)
         self.orc = oracle.OracleCache(w.n_seq, w.n_kv_heads, w.group_size, w.head_dim, w.hash_bits, self.gpu.Cmax,
                                       w.budgets(), w.dtype, n_sink=w.n_sink, n_recent=w.n_recent, threads=8)
         self.dK, self.dQ, self.dV = to_dev(self.K, w), to_dev(self.Q, w), to_dev(self.V, w)

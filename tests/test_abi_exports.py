@@ -40,7 +40,8 @@ def test_host_side_validation_needs_no_gpu():
 def test_flag_values_match_the_header_and_packed_layout_is_validated_on_the_host():
     text = open(os.path.join(ROOT, "include", "hashevict.h")).read()
     flags = {m.group(1): int(m.group(2)) for m in re.finditer(r"#define\s+(HE_FLAG_[A-Z_]+)\s+(\d+)u", text)}
-    assert flags == {"HE_FLAG_WRITE_SCORES": binding.HE_FLAG_WRITE_SCORES, "HE_FLAG_PACKED_CODES": binding.HE_FLAG_PACKED_CODES}
+    assert flags == {"HE_FLAG_WRITE_SCORES": binding.HE_FLAG_WRITE_SCORES, "HE_FLAG_PACKED_CODES": binding.HE_FLAG_PACKED_CODES,
+                     "HE_FLAG_EARLY_INPUTS": binding.HE_FLAG_EARLY_INPUTS}
     L = binding.lib()
     packed = binding.HE_FLAG_PACKED_CODES
     ca = binding.he_cache()
