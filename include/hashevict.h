@@ -9,7 +9,8 @@
  *
  * General rules for every entry point
  *   - All tensor pointers are DEVICE pointers owned by the caller unless a parameter says "host".
- *     The library allocates no memory; scratch space is passed in by the caller.
+ *     The library allocates no memory; scratch space is passed in by the caller (the one exception,
+ *     he_prefill_compress_noalloc, uses an array that is part of the library's device image).
  *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*) and return at once;
  *     they never synchronise (the *_host variants are the exception and say so). Results are
  *     valid once the stream has been synchronised.
@@ -28,7 +29,11 @@
  *                                         two layouts are the same bytes.
  *   scores            [B, Hkv, Cmax]      fp32, -(Hamming distance summed over the group)
  *   pos               [B, Hkv, Cmax]      int32 token position held by the slot, -1 = empty
- *   budget            [B]                 int32 C_s <= Cmax, read-only
+ *   budget            [B]                 int32, 1 <= C_s <= Cmax, read-only. Checked on the host only when
+ *                                         he_cache.budget_host is given (HE_ERR_INVALID_ARG); on the device a value
+ *                                         above Cmax counts as Cmax and a value below 1 as "this sequence stores
+ *                                         nothing" (prefill leaves its units empty, decode leaves them untouched and
+ *                                         reports victim -1).
  *   fill, next_pos    [B, Hkv]            int32 valid slots / position of the next token, per unit
  *   W                 [d, b]              fp32 row-major: W = R^T of Eq. 2, read-only while in use
  */
@@ -135,10 +140,15 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
 /*
  * he_prefill_compress - "Prompt Encoding Stage": the cache is reset, the first C_s prompt tokens fill
  * slots 0..C_s-1, and every later prompt token t = C_s..N_s-1 goes through Algorithm 1 in order, so
- * the result equals he_reset followed by N_s calls of he_decode_step.
+ * the result equals he_reset followed by N_s calls of he_decode_step - given the same hash bits. The bulk
+ * projection of the prompt (tensor cores for bf16 rows) and the projection inside a decode step round the same sum
+ * differently, so a bit whose exact projection lies within 1e-5 * |x| * |w| of zero (about one in 1e4 to 1e5 bits)
+ * may come out differently on the two routes, and the two caches then part ways from that token on; each route on
+ * its own is a valid run of Algorithm 1 under Eq. 2's tolerance.
  * q: [B, Hkv*G, N, d], k, v: [B, Hkv, N, d] addressed with element strides (batch, head, token);
  * channels are contiguous and every row is 16-byte aligned. prompt_len: [B] int32 on the device,
- * each <= max_prompt_len. Queries of tokens that are appended are never read.
+ * each <= max_prompt_len (a larger value counts as max_prompt_len, a negative one as 0). Queries of tokens that
+ * are appended are never read.
  * workspace: at least he_workspace_bytes(cfg, max_prompt_len) bytes, 256-byte aligned; it receives
  * the prompt codes: key codes [B*Hkv, Nmax, Wd] followed by query codes [B*Hkv, Nmax, G, Wd]
  * (query codes of appended tokens are left unwritten). scores hold the last evicting step's values.
@@ -147,7 +157,8 @@ int he_prefill_compress(const he_config* cfg, const he_cache* cache, const void*
                         const int64_t q_strides[3], const int64_t kv_strides[3], const int32_t* prompt_len,
                         int32_t max_prompt_len, void* workspace, size_t workspace_bytes, void* stream);
 
-/* Bytes of he_cache.step_scratch: the codes of one decode step's new rows, (G + 1) * Wd words per unit (0 on bad input). */
+/* Bytes of he_cache.step_scratch: the codes of one decode step's new rows, (G + 1) * Wd words per unit, plus the
+   three-term bf16 image of W that the bulk projection kernels read (0 on bad input). */
 size_t he_step_scratch_bytes(const he_config* cfg);
 
 /* Scratch bytes he_prefill_compress needs for prompts of up to max_prompt_len tokens (0 on bad input). */
@@ -279,8 +290,12 @@ int he_prefill_compress_noalloc(const he_config* cfg, const he_cache* cache, con
 /*
  * he_device_error_count - how many thread blocks of this library's kernels gave up on a bounded device-side
  * wait since the library was loaded (0 in a healthy process; the kernels never wait without a limit, and a
- * block that hits one releases what it holds and returns). This call synchronises the device. Returns -1 if the
- * counter cannot be read. Diagnostic only: the paper has no counterpart.
+ * block that hits one releases what it holds and returns), plus, in the bounds-checking debug build, how many
+ * indices were found out of range. A call during which the counter rose has returned HE_OK all the same (calls
+ * only enqueue work), but its outputs are undefined: he_hash_keys, he_prefill_compress and its variants, and
+ * he_decode_step with a step scratch are the calls whose kernels contain such waits. This is the one call of the
+ * library, besides the *_host variants, that synchronises the device. Returns -1 if the counter cannot be read.
+ * Diagnostic only: the paper has no counterpart.
  */
 int he_device_error_count(void);
 

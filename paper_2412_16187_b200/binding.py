@@ -49,7 +49,10 @@ def lib():
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.build_cuda() if not os.path.exists(_build.LIB_PATH) else _build.LIB_PATH
+    if os.environ.get("HE_DEBUG_LIB") == "1":  # the bounds-checking build (see build.build_cuda)
+        path = _build.build_cuda(debug=True)
+    else:
+        path = _build.build_cuda() if not os.path.exists(_build.LIB_PATH) else _build.LIB_PATH
     try:
         L = ctypes.CDLL(path)
     except OSError as e:  # no silent fallback

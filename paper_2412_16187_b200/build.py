@@ -22,14 +22,22 @@ def nvcc_path() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
-def build_cuda(force: bool = False, verbose: bool = False) -> str:
-    """Compile csrc/*.cu into libhashevict.so; rebuilds only when a source or header is newer."""
+DEBUG_LIB_PATH = os.path.join(_PKG, "libhashevict_debug.so")
+
+
+def build_cuda(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile csrc/*.cu into libhashevict.so; rebuilds only when a source or header is newer.
+
+    debug=True builds libhashevict_debug.so with -DHE_BOUNDS_CHECK instead: every slot and token index is range-checked
+    before it is used as an address, a failed check skips the access and raises he_device_error_count(). The binding
+    loads that library when HE_DEBUG_LIB=1 is set before the first call."""
+    out = DEBUG_LIB_PATH if debug else LIB_PATH
     deps = _SOURCES + _HEADERS
-    if not force and os.path.exists(LIB_PATH) and all(os.path.getmtime(LIB_PATH) >= os.path.getmtime(p) for p in deps):
-        return LIB_PATH
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
-    cmd = [nvcc_path()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+    if not force and os.path.exists(out) and all(os.path.getmtime(out) >= os.path.getmtime(p) for p in deps):
+        return out
+    tmp = out + f".tmp{os.getpid()}"
+    cmd = [nvcc_path()] + NVCC_FLAGS + (["-DHE_BOUNDS_CHECK"] if debug else []) + (["-Xptxas", "-v"] if verbose else []) + \
         ["-I", os.path.join(_ROOT, "include"), "-o", tmp] + _SOURCES
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, out)
+    return out

@@ -42,6 +42,31 @@ __device__ __forceinline__ void store_slot_code(const he_config& cfg, uint32_t* 
   }
 }
 
+// Device-side trouble counter behind he_device_error_count: CTAs that gave up on a bounded wait and, in a build with
+// -DHE_BOUNDS_CHECK, indices found out of range (stays 0 in a healthy run).
+__device__ int g_tc_error = 0;
+
+// Bounds checks of the debug build (build_cuda(debug=True) -> libhashevict_debug.so). Every slot or token index that a
+// kernel computes or reads from memory before using it as an address goes through HE_IN_RANGE(i, n): true when
+// 0 <= i < n. In the debug build a failed check is counted and the caller skips the access, so the kernel finishes
+// and the host reads the count; the release build compiles the test away.
+#ifdef HE_BOUNDS_CHECK
+__device__ __forceinline__ bool he_in_range(long long i, long long n) {
+  if (i >= 0 && i < n) return true;
+  atomicAdd(&g_tc_error, 1);
+  return false;
+}
+#define HE_IN_RANGE(i, n) ::he::he_in_range((long long)(i), (long long)(n))
+#else
+#define HE_IN_RANGE(i, n) true
+#endif
+
+// Device-side inputs the host cannot see are clamped where they are read: a prompt length into [0, Nmax] (the
+// prompt-code scratch holds Nmax rows per unit), a budget into [0, Cmax]. A budget below 1 leaves nothing to store:
+// the prefill calls then treat the sequence as empty and the decode calls leave its units untouched.
+__device__ __forceinline__ int clamp_budget(int c, int cmax) { return min(max(c, 0), cmax); }
+__device__ __forceinline__ int clamp_len(int n, int nmax, int c) { return c < 1 ? 0 : min(max(n, 0), nmax); }
+
 __device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
 
 __device__ __forceinline__ uint32_t word_mask(int b, int w) {

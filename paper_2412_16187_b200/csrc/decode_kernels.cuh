@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? (PRE ? 6 : 4) : 1)) decode_st
     const char* src = static_cast<const char*>(is_k ? a.k : a.v) + (size_t)unit * d * es;
     rowreg = __ldg(reinterpret_cast<const uint4*>(src) + (is_k ? tid : tid - cpr));
   }
-  const int C = min(a.n_budget_vals > 0 ? a.budget_vals[s] : a.ca.budget[s], Cmax);
+  const int C = clamp_budget(a.n_budget_vals > 0 ? a.budget_vals[s] : a.ca.budget[s], Cmax);
   const int fill = a.ca.fill[unit];
   const int t = a.ca.next_pos[unit];
 
@@ -234,7 +234,7 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? (PRE ? 6 : 4) : 1)) decode_st
   if (a.qcodes_out != nullptr && tid < G * WORDS) a.qcodes_out[(size_t)unit * G * WORDS + tid] = codes_s[tid];
 
   // (3) Eq. 5 / Eq. 6
-  const bool evict = fill >= C;
+  const bool evict = C >= 1 && fill >= C;
   int slot = fill;
   if (evict) {
     Ctx ctx;
@@ -376,6 +376,13 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? (PRE ? 6 : 4) : 1)) decode_st
   }
 
   if (!evict) cp_async_wait_all();  // a unit that is still filling never looked at the copied table
+  if (C < 1 || !HE_IN_RANGE(slot, C)) {  // a unit without a budget holds nothing: report it and leave the state alone
+    if (tid == 0) {
+      a.victim_out[unit] = -1;
+      if (a.evicted_pos_out != nullptr) a.evicted_pos_out[unit] = -1;
+    }
+    return;
+  }
   // (4) Algorithm 1 lines 2-5: the slot takes the new token's K, V, code and position
   const size_t slot_idx = (size_t)unit * Cmax + slot;
   if (tid < 2 * cpr) {

@@ -512,7 +512,7 @@ __global__ void __launch_bounds__(kSmThreads, 2) decode_step_sm_kernel(const Dec
       if (j == i) fill = fl[j], t = tt[j];
     const SmUnit& u = su[i];
     const int C = u.C;
-    if (C < 1) {  // a unit without a budget holds nothing: report it and leave the state alone
+    if (C < 1 || !HE_IN_RANGE(fill, Cmax + 1)) {  // a unit without a budget holds nothing: report it and leave the state alone
       if (lane == 0) {
         *u.victim_p = -1;
         if (u.evpos_p != nullptr) *u.evpos_p = -1;
@@ -529,6 +529,7 @@ __global__ void __launch_bounds__(kSmThreads, 2) decode_step_sm_kernel(const Dec
       }
       slot = min((int)(kKeyIdxMask - (fin & kKeyIdxMask)), C - 1);  // (the clamp never acts on a scored table)
     }
+    if (!HE_IN_RANGE(slot, C)) return;
     const size_t row_bytes = (size_t)cpr * 16;
     for (int c = lane; c < 2 * cpr; c += 32) {
       const bool is_k = c < cpr;

@@ -47,8 +47,8 @@ __global__ void __launch_bounds__(kHashThreads) hash_rows_kernel(const HashJob j
   } else {
     const int seg = blockIdx.y;
     const int s = seg / job.heads, hh = seg % job.heads;
-    const long long N = job.prompt_len[s];
-    const long long C = job.budget[s];
+    const long long C = max(job.budget[s], 0);
+    const long long N = clamp_len(job.prompt_len[s], job.Nmax, (int)min(C, 1LL));
     base = static_cast<const char*>(job.x) + (s * job.s0 + hh * job.s1) * es;
     stride = job.s2;
     r_end = N;

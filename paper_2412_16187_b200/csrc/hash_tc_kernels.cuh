@@ -32,7 +32,6 @@ constexpr int kTcLag = 2;             // cp.async groups the producer leaves in 
 constexpr uint32_t kTcSpinLimit = 1u << 22;
 constexpr int kTcLenCache = 2048;     // sequences whose prompt length and budget are cached in shared memory
 
-__device__ int g_tc_error = 0;  // number of CTAs that gave up on a bounded wait (stays 0 in a healthy run)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -216,8 +215,8 @@ __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long lo
   } else {
     const int s = nseq_dense > 0 ? s_d : seg / job.heads, hh = nseq_dense > 0 ? hh_d : seg % job.heads;
     // lengths come from the CTA's shared-memory copy when the batch fits it: skipping an empty tile is then cheap
-    const long long N = s < kTcLenCache ? s_len[s] : job.prompt_len[s];
-    const long long C = s < kTcLenCache ? s_bud[s] : job.budget[s];
+    const long long C = s < kTcLenCache ? s_bud[s] : max(job.budget[s], 0);
+    const long long N = s < kTcLenCache ? s_len[s] : clamp_len(job.prompt_len[s], job.Nmax, (int)min(C, 1LL));
     o->c2 = hh;
     o->c3 = s;
     o->base = static_cast<const char*>(job.x) + (s * job.s0 + hh * job.s1) * 2;
@@ -297,8 +296,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   const int nseq = job.mode != 0 ? (int)(total_tiles / tiles_per_seg) / job.heads : 0;
   if (job.mode != 0) {
     for (int i = threadIdx.x; i < nseq && i < kTcLenCache; i += kTcThreads) {
-      s_len[i] = job.prompt_len[i];
-      s_bud[i] = job.budget[i];
+      s_bud[i] = max(job.budget[i], 0);
+      s_len[i] = clamp_len(job.prompt_len[i], job.Nmax, min(s_bud[i], 1));
     }
   }
   if (tid == 0) s_nseq_dense = 0;

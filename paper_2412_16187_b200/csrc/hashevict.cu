@@ -1,13 +1,18 @@
 // HashEvict eviction hot path for B200 (sm_100a): host side of the C ABI declared in include/hashevict.h.
 //
 // The kernels live in the .cuh files next to this one:
-//   hash_kernels.cuh     Eq. 2 on many rows (he_hash_keys, phase 1 of he_prefill_compress)
-//   decode_kernels.cuh   Algorithm 1 lines 1-5 for one unit per CTA (he_decode_step)
-//   prefill_kernels.cuh  the prompt-encoding replay and the K/V gather (phases 2, 3 of he_prefill_compress)
+//   hash_kernels.cuh, hash_tc_kernels.cuh   Eq. 2 on many rows (he_hash_keys, phase 1 of he_prefill_compress)
+//   decode_kernels.cuh, decode_sm_kernels.cuh   Algorithm 1 lines 1-5 (he_decode_step)
+//   prefill_kernels.cuh, prefill_tc_kernels.cuh   the prompt-encoding replay and the K/V gather (phases 2, 3 of
+//                                                 he_prefill_compress)
 //
-// One projection order is used by every path (bulk hash, decode, prefill) so that they produce the same bits:
-// channels are cut into chunks of 32; a chunk's partial sum is an fmaf chain in ascending channel order starting
-// from 0; the partial sums are added in ascending chunk order; the bit is (sum >= 0).
+// Eq. 2 is evaluated in one of two ways. CUDA cores (fp32 rows, odd head sizes, small calls, the per-unit decode
+// kernel): channels are cut into chunks of 32; a chunk's partial sum is an fmaf chain in ascending channel order
+// starting from 0; the partial sums are added in ascending chunk order; the bit is (sum >= 0). Tensor cores (bf16
+// rows in bulk, and the one-CTA-per-SM decode kernel): W as three bf16 terms whose sum is W exactly, every product
+// exact, fp32 accumulation in the instruction's own order. Both stay far inside the tolerance of Eq. 2's contract (a
+// bit may differ from exact arithmetic only where the exact projection is within 1e-5 * |x| * |w| of zero), but they
+// are two roundings of the same sum: for such a borderline bit two paths may disagree with each other.
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -100,6 +105,15 @@ int check_cache(const he_cache* ca) {
     return fail(HE_ERR_INVALID_ARG, "cache has a null pointer");
   if (!aligned16(ca->k_cache) || !aligned16(ca->v_cache) || !aligned16(ca->codes) || !aligned16(ca->scores) || !aligned16(ca->pos))
     return fail(HE_ERR_INVALID_ARG, "cache arrays must be 16-byte aligned");
+  return HE_OK;
+}
+
+// Budgets must lie in [1, max_budget]; the host can only check them when the caller gave a mirror.
+int check_budget_mirror(const he_config* cfg, const he_cache* ca) {
+  if (ca->budget_host == nullptr) return HE_OK;
+  for (int s = 0; s < cfg->batch; ++s)
+    if (ca->budget_host[s] < 1 || ca->budget_host[s] > cfg->max_budget)
+      return fail(HE_ERR_INVALID_ARG, "budget %d of sequence %d outside [1, max_budget = %d]", ca->budget_host[s], s, cfg->max_budget);
   return HE_OK;
 }
 
@@ -534,6 +548,7 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
   if (int rc = check_cache(cache)) return rc;
   if (!q || !k || !v || !victim_out) return fail(HE_ERR_INVALID_ARG, "q, k, v or victim_out is null");
   if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return fail(HE_ERR_INVALID_ARG, "q, k, v must be 16-byte aligned");
+  if (int rc = check_budget_mirror(cfg, cache)) return rc;
   const int Wd = words_of(cfg->hash_bits);
   const int cb = packed_code_bytes(*cfg);  // 1..3 bytes per slot, or 0: word layout
   const long long nvec = cb ? ((long long)cfg->max_budget * cb + 15) / 16 : ((long long)cfg->max_budget * Wd + 3) / 4;
@@ -648,6 +663,7 @@ int prefill_impl(int variant /* 0: Algorithm 1, 1: averaged Hamming, 2: L2 norm 
   if (!q || !k || !v || !q_strides || !kv_strides || !prompt_len || !workspace)
     return fail(HE_ERR_INVALID_ARG, "q, k, v, strides, prompt_len or workspace is null");
   if (max_prompt_len < 0) return fail(HE_ERR_INVALID_ARG, "max_prompt_len %d < 0", max_prompt_len);
+  if (int rc = check_budget_mirror(cfg, cache)) return rc;
   const int es = esize_of(cfg->dtype);
   for (int i = 0; i < 3; ++i)
     if ((q_strides[i] * es) % 16 != 0 || (kv_strides[i] * es) % 16 != 0)
@@ -727,7 +743,7 @@ int prefill_impl(int variant /* 0: Algorithm 1, 1: averaged Hamming, 2: L2 norm 
   }
 
   // phase 3: surviving K / V rows into their slots
-  GatherArgs ga{*cfg, *cache, k, v, kv_strides[0], kv_strides[1], kv_strides[2]};
+  GatherArgs ga{*cfg, *cache, k, v, kv_strides[0], kv_strides[1], kv_strides[2], max_prompt_len};
   const long long per_unit = 2LL * cfg->max_budget * (cfg->head_dim * es / 16);
   const long long gx = (per_unit + kGatherThreads * kGatherUnroll - 1) / (kGatherThreads * kGatherUnroll);
   if (units > 65535) return fail(HE_ERR_UNSUPPORTED, "more than 65535 units in one prefill call");

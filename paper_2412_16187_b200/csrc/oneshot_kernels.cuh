@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kOneshotThreads) key_norms_kernel(const NormAr
   const long long unit = blockIdx.y;
   const int s = (int)(unit / a.cfg.n_kv_heads), h = (int)(unit % a.cfg.n_kv_heads);
   const int i = blockIdx.x * kOneshotThreads + threadIdx.x;
-  if (i >= a.prompt_len[s]) return;
+  if (i >= min(a.prompt_len[s], (int)a.Nmax)) return;
   const int d = a.cfg.head_dim, es = esize_of(a.cfg.dtype);
   const char* row = static_cast<const char*>(a.k) + (s * a.s0 + h * a.s1 + (long long)i * a.s2) * es;
   float acc = 0.f;
@@ -91,8 +91,8 @@ __global__ void __launch_bounds__(kOneshotThreads) oneshot_rank_kernel(const One
   const int s = (int)(unit / cfg.n_kv_heads);
   const int G = cfg.group_size, GW = G * WORDS;
   const long long Cmax = cfg.max_budget;
-  const int C = min(a.ca.budget[s], (int)Cmax);
-  const int N = a.prompt_len[s];
+  const int C = clamp_budget(a.ca.budget[s], (int)Cmax);
+  const int N = clamp_len(a.prompt_len[s], a.Nmax, C);
   const int keep = N < C ? N : C;
   const uint32_t* kc_u = a.kcodes + unit * a.Nmax * WORDS;
   const uint32_t* qc_u = a.qcodes + unit * a.Nmax * GW;
@@ -268,8 +268,15 @@ __global__ void __launch_bounds__(kStepL2Threads) decode_step_l2_kernel(const St
   const long long unit = (long long)blockIdx.y * cfg.n_kv_heads + blockIdx.x;
   const int d = cfg.head_dim, es = esize_of(cfg.dtype), Wd = (cfg.hash_bits + 31) / 32;
   const long long Cmax = cfg.max_budget;
-  const int C = min(a.ca.budget[blockIdx.y], (int)Cmax);
-  const int fill = a.ca.fill[unit], t = a.ca.next_pos[unit];
+  const int C = clamp_budget(a.ca.budget[blockIdx.y], (int)Cmax);
+  const int fill = min(a.ca.fill[unit], C), t = a.ca.next_pos[unit];
+  if (C < 1) {  // a unit without a budget holds nothing: report it and leave the state alone
+    if (tid == 0) {
+      a.victim_out[unit] = -1;
+      if (a.evicted_pos_out != nullptr) a.evicted_pos_out[unit] = -1;
+    }
+    return;
+  }
   const char* kr = static_cast<const char*>(a.k) + unit * d * es;
   const char* vr = static_cast<const char*>(a.v) + unit * d * es;
   if (tid == 0) {
@@ -307,6 +314,7 @@ __global__ void __launch_bounds__(kStepL2Threads) decode_step_l2_kernel(const St
   } else {
     __syncthreads();
   }
+  if (!HE_IN_RANGE(slot, C)) return;
   const long long dst = unit * Cmax + slot;
   for (int i = tid; i < 2 * (d * es / 16); i += kStepL2Threads) {
     const int half = d * es / 16;

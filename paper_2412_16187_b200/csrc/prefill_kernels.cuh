@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const h
     unsigned long long key = 0ull;
     if (i < units) {
       const int s = i / cfg.n_kv_heads;
-      const long long C = budget[s], N = prompt_len[s];
+      const long long C = clamp_budget(budget[s], cfg.max_budget), N = clamp_len(prompt_len[s], 0x7FFFFFFF, (int)C);
       const long long work = N > C ? (N - C) * (C + step_cost) + 1 : 1;  // evicting steps x (slots scanned + fixed cost)
       key = ((unsigned long long)work << 20) | (unsigned long long)(0xFFFFF - i);
     }
@@ -249,8 +249,8 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : (NT <= 512 ? 2 : 1))) pre
     const long long unit = s_unit;
     if (unit < 0) break;
     const int s = (int)(unit / cfg.n_kv_heads);
-    const int C = min(a.ca.budget[s], (int)Cmax);
-    const int N = a.prompt_len[s];
+    const int C = clamp_budget(a.ca.budget[s], (int)Cmax);
+    const int N = clamp_len(a.prompt_len[s], a.Nmax, C);
     const int fill0 = N < C ? N : C;
     const uint32_t* kc_u = a.kcodes + unit * a.Nmax * WORDS;
     const uint32_t* qc_u = a.qcodes + unit * a.Nmax * G * WORDS;
@@ -339,7 +339,7 @@ __global__ void __launch_bounds__(NT, (NT <= 256 ? 4 : (NT <= 512 ? 2 : 1))) pre
           if (fin_el != 0u) fin = fin_el;
         }
         const int slot = (int)(kKeyIdxMask - (fin & kKeyIdxMask));
-        if (slot % NT == tid) {  // the slot's own scanning thread rewrites it, so no extra barrier is needed
+        if (slot % NT == tid && HE_IN_RANGE(slot, C)) {  // the slot's own scanning thread rewrites it, so no extra barrier is needed
           const int rr = slot / NT;
 #pragma unroll
           for (int r = 0; r < SPT; ++r)
@@ -399,8 +399,8 @@ __global__ void prefill_replay_smem_kernel(const ReplayArgs a) {
   const int s = (int)(unit / cfg.n_kv_heads);
   const int G = cfg.group_size;
   const long long Cmax = cfg.max_budget;
-  const int C = a.ca.budget[s];
-  const int N = a.prompt_len[s];
+  const int C = clamp_budget(a.ca.budget[s], (int)Cmax);
+  const int N = clamp_len(a.prompt_len[s], a.Nmax, C);
   const int fill0 = N < C ? N : C;
   uint32_t* codes_s = rsm;                                                           // [smem_slots][WORDS]
   int32_t* pos_s = reinterpret_cast<int32_t*>(rsm + (size_t)a.smem_slots * WORDS);  // [smem_slots]
@@ -458,7 +458,7 @@ __global__ void prefill_replay_smem_kernel(const ReplayArgs a) {
         if (fin_el != 0u) fin = fin_el;
       }
       const int slot = (int)(kKeyIdxMask - (fin & kKeyIdxMask));
-      if (slot % NT == tid) {
+      if (slot % NT == tid && HE_IN_RANGE(slot, C)) {
 #pragma unroll
         for (int w = 0; w < WORDS; ++w) codes_s[slot * WORDS + w] = rec[Ctx::kRecWords + w];
         pos_s[slot] = t;
@@ -497,6 +497,7 @@ struct GatherArgs {
   const void* k;
   const void* v;
   long long s0, s1, s2;
+  long long Nmax;  // prompt tokens per unit in k, v
 };
 
 constexpr int kGatherThreads = 256;
@@ -509,7 +510,7 @@ __global__ void __launch_bounds__(kGatherThreads) prefill_gather_kernel(const Ga
   const int s = (int)(unit / cfg.n_kv_heads), h = (int)(unit % cfg.n_kv_heads);
   const int d = cfg.head_dim, es = esize_of(cfg.dtype);
   const long long Cmax = cfg.max_budget;
-  const int fill = a.ca.fill[unit];
+  const int fill = min(max(a.ca.fill[unit], 0), (int)Cmax);
   const int cpr = d * es / 16;
   const long long ntask = 2LL * fill * cpr;
   const long long base = (long long)blockIdx.x * kGatherThreads * kGatherUnroll;
@@ -526,6 +527,7 @@ __global__ void __launch_bounds__(kGatherThreads) prefill_gather_kernel(const Ga
       const long long rem = task % ((long long)fill * cpr);
       const int j = (int)(rem / cpr), ch = (int)(rem % cpr);
       const long long tok = pp[j];
+      if (!HE_IN_RANGE(tok, a.Nmax)) continue;  // (a slot of a valid cache names a prompt token)
       const char* src = static_cast<const char*>(which ? a.v : a.k) + (s * a.s0 + h * a.s1 + tok * a.s2) * es;
       val[i] = __ldg(reinterpret_cast<const uint4*>(src) + ch);
       dst_off[i] = (((unit * Cmax + j) * d * es) / 16 + ch) * 2 + which;

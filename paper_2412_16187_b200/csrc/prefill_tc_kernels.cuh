@@ -242,8 +242,8 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     const long long unit = s_unit;
     if (unit < 0) break;
     const int s = (int)(unit / cfg.n_kv_heads);
-    const int C = min(a.ca.budget[s], (int)Cmax);
-    const int N = a.prompt_len[s];
+    const int C = clamp_budget(a.ca.budget[s], (int)Cmax);
+    const int N = clamp_len(a.prompt_len[s], a.Nmax, C);
     const int fill0 = N < C ? N : C;
     const uint32_t* kc_u = a.kcodes + unit * a.Nmax * WORDS;
     const uint32_t* qc_u = a.qcodes + unit * a.Nmax * G * WORDS;
@@ -668,10 +668,12 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             vb3 = (mine && sel == 3) ? nv : (k3 == best ? kAbsent : vb3);
             // Algorithm 1 lines 2-5 on the table (K / V rows follow in the gather kernel). Every lane stores the same
             // values to the same addresses: no divergent branch, and each lane later reads back its own stores.
-            owner[slot] = (int16_t)r;
+            if (HE_IN_RANGE(slot, C)) {
+              owner[slot] = (int16_t)r;
 #pragma unroll
-            for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
-            pos_t[slot] = t0 + r;
+              for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
+              pos_t[slot] = t0 + r;
+            }
             if (slot == kRtIdxMask - (kb_n & kRtIdxMask)) own_n = r;  // the owner fetched ahead predates this step
             dd = dd_n, kb = kb_n, own_kb = own_n;
 #pragma unroll
@@ -763,10 +765,12 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
               // finish step r here, then stop
               const int best = max(kb, kn);
               const int slot = kRtIdxMask - (best & kRtIdxMask);
-              owner[slot] = (int16_t)r;
+              if (HE_IN_RANGE(slot, C)) {
+                owner[slot] = (int16_t)r;
 #pragma unroll
-              for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
-              pos_t[slot] = t0 + r;
+                for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
+                pos_t[slot] = t0 + r;
+              }
               if (PROT && GLOBAL_TABLE && lane == ((t0 + r) & 31)) myring = slot;
               done = r + 1;
               break;

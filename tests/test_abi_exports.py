@@ -54,3 +54,20 @@ def test_flag_values_match_the_header_and_packed_layout_is_validated_on_the_host
     # 32- and 64-bit codes are the same bytes in both layouts: the flag changes nothing, the null cache is what fails
     same = binding.he_config(1, 1, 1, 128, 64, 36, 0, 0, 1, packed)
     assert L.he_reset(ctypes.byref(same), ctypes.byref(ca), None) == 1 and b"null" in L.he_last_error()
+
+
+def test_budgets_outside_the_cache_are_rejected_on_the_host_when_a_mirror_is_given():
+    """Budgets must lie in [1, max_budget]; with he_cache.budget_host the call fails before anything is launched
+    (the pointers below are never dereferenced: the check comes first)."""
+    L = binding.lib()
+    cfg = binding.he_config(2, 2, 4, 128, 64, 64, 0, 0, 1, 1)
+    fake = 0x10000
+    for bad, word in (([0, 8], b"budget 0"), ([8, -3], b"budget -3"), ([8, 65], b"budget 65")):
+        mirror = (ctypes.c_int32 * 2)(*bad)
+        ca = binding.he_cache(*([fake] * 9), ctypes.cast(mirror, ctypes.c_void_p), None)
+        rc = L.he_decode_step(ctypes.byref(cfg), ctypes.byref(ca), fake, fake, fake, fake, None, None, None)
+        assert rc == 1 and word in L.he_last_error(), L.he_last_error()
+        i64x3 = ctypes.c_int64 * 3
+        rc = L.he_prefill_compress(ctypes.byref(cfg), ctypes.byref(ca), fake, fake, fake, i64x3(128, 128, 128), i64x3(128, 128, 128),
+                                   fake, 16, 0x20000, 1 << 30, None)
+        assert rc == 1 and word in L.he_last_error(), L.he_last_error()

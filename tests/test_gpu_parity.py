@@ -172,7 +172,7 @@ def test_enqueued_host_steps_on_two_streams_match_device_calls():
             assert torch.equal(getattr(ref.gpu, name), getattr(c.gpu, name)), name
 
 
-def _sampled_full_size_check(w, seqs, decode_steps):
+def _sampled_full_size_check(w, seqs, decode_steps, early_inputs=False):
     """Full-size workload on the device in the launch configuration the benchmark times; the oracle replays only
     the sampled sequences (all their KV heads) on the device's codes and must reproduce their final state."""
     import oracle as orc
@@ -181,7 +181,7 @@ def _sampled_full_size_check(w, seqs, decode_steps):
     W = wl.gen_W(w)
     plen, budgets = w.prompt_lens(), w.budgets()
     gpu = HashEvictCache(w.n_seq, w.n_kv_heads, w.group_size, w.head_dim, w.hash_bits, budgets, torch.from_numpy(W),
-                         dtype=torch_dtype(w))
+                         dtype=torch_dtype(w), early_inputs=early_inputs)
     tdt = torch_dtype(w)
     dK = torch.zeros((w.n_seq, w.n_kv_heads, Nmax, w.head_dim), dtype=tdt, device="cuda")
     dV = torch.zeros_like(dK)
@@ -229,17 +229,32 @@ def _sampled_full_size_check(w, seqs, decode_steps):
 
 
 def test_full_size_throughput_batch_sampled_sequences():
+    """Configuration 5 in full on the device; the oracle follows 8 of the 64 sequences (shortest, median and longest
+    budget plus five seeded picks) through the prefill and 64 decode steps."""
     w = wl.CONFIGS["throughput_batch"]
     b = w.budgets()
-    order = np.argsort(b)
-    _sampled_full_size_check(w, [int(order[0]), int(order[len(order) // 2]), int(order[-1])], decode_steps=4)
+    order = np.argsort(b, kind="stable")
+    picks = [int(order[0]), int(order[len(order) // 2]), int(order[-1])]
+    rng = np.random.default_rng(5)
+    for s in rng.permutation(w.n_seq):
+        if len(picks) == 8:
+            break
+        if int(s) not in picks:
+            picks.append(int(s))
+    _sampled_full_size_check(w, picks, decode_steps=64)
+
+
+def test_full_size_throughput_batch_sampled_sequences_early_inputs():
+    w = wl.CONFIGS["throughput_batch"]
+    order = np.argsort(w.budgets(), kind="stable")
+    _sampled_full_size_check(w, [int(order[1]), int(order[-2])], decode_steps=24, early_inputs=True)
 
 
 def test_full_size_long_prefill_sampled_layer():
     # full per-unit size (32768-token prompt, 9830 slots, 22938 evicting steps), 4 of the 32 folded layers on the
-    # device, one of them replayed by the oracle
+    # device, two of them replayed by the oracle, 16 decode steps
     w = wl.CONFIGS["long_prefill"].scaled(layers=4)
-    _sampled_full_size_check(w, [2], decode_steps=3)
+    _sampled_full_size_check(w, [1, 2], decode_steps=16)
 
 
 def test_prefill_with_token_major_strided_inputs():

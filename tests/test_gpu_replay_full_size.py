@@ -1,4 +1,4 @@
-"""Full-size cross-check of the replay implementations: at BASELINE sizes the oracle can only follow sampled units
+"""Full-size cross-check of the replay implementations: at the full workload sizes the oracle follows sampled units
 (tests/test_gpu_parity.py does that), so here the tensor-core replay (8-bit and bf16 operands) and the CUDA-core
 replay, each of which is checked against the oracle on smaller shapes, must leave bit-identical caches on the whole
 throughput_batch workload (also with the paper's protected windows) and on four layers of long_prefill (9830-slot

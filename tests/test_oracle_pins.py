@@ -499,3 +499,43 @@ def test_l2_decode_steps_keep_the_lowest_norms_and_the_newest_token():
                 n2 = (ks[:T - 1, 0, h].astype(np.float64) ** 2).sum(1)
                 want = set(np.argsort(n2, kind="stable")[:C - 1].tolist()) | {T - 1}
                 assert set(oc.pos[0, h].tolist()) == want
+
+
+def test_prefill_follows_the_strides_of_token_major_inputs():
+    """The prompt tensors may be strided views (token-major storage, as a fused QKV projection leaves them; a slice of
+    a longer buffer): the oracle must read the same tokens as from contiguous copies. Both the embedding route and the
+    code route, with ragged prompts so that a wrong stride lands on another token's row."""
+    rng = np.random.default_rng(7)
+    B, H, G, d, b, N, C = 2, 3, 2, 16, 12, 40, 9
+    W = rng.standard_normal((d, b)).astype(np.float32)
+    # token-major storage [B, N + 5, heads, d], seen as [B, heads, N, d] through a transpose and a slice
+    Kt = rng.standard_normal((B, N + 5, H, d)).astype(np.float32)
+    Vt = rng.standard_normal((B, N + 5, H, d)).astype(np.float32)
+    Qt = rng.standard_normal((B, N + 5, H * G, d)).astype(np.float32)
+    Kv, Vv, Qv = (x[:, 2:N + 2].transpose(0, 2, 1, 3) for x in (Kt, Vt, Qt))
+    assert not Kv.flags.c_contiguous and Kv.strides[2] == H * d * 4
+    plen = np.array([N, 23], dtype=np.int32)
+    budgets = np.array([C, 7], dtype=np.int32)
+
+    def run(q, k, v):
+        oc = oracle.OracleCache(B, H, G, d, b, 12, budgets, "f32", n_sink=1, n_recent=2, threads=2)
+        oc.prefill(W, q, k, v, plen)
+        return oc
+
+    a = run(Qv, Kv, Vv)
+    c = run(np.ascontiguousarray(Qv), np.ascontiguousarray(Kv), np.ascontiguousarray(Vv))
+    for name in ("codes", "pos", "fill", "next_pos", "scores", "k_cache", "v_cache"):
+        assert np.array_equal(getattr(a, name), getattr(c, name)), name
+    # the code route: codes hashed from the contiguous copies, K / V handed over as the strided views
+    kc = np.stack([oracle.hash_rows(np.ascontiguousarray(Kv[s]).reshape(-1, d), W, "f32").reshape(H, N, -1) for s in range(B)])
+    qc = np.stack([oracle.hash_rows(np.ascontiguousarray(Qv[s]).reshape(-1, d), W, "f32").reshape(H, G, N, -1).transpose(0, 2, 1, 3)
+                   for s in range(B)])
+    e = oracle.OracleCache(B, H, G, d, b, 12, budgets, "f32", n_sink=1, n_recent=2, threads=2)
+    e.prefill_codes(np.ascontiguousarray(kc), np.ascontiguousarray(qc), Kv, Vv, plen)
+    for name in ("codes", "pos", "fill", "next_pos", "scores", "k_cache", "v_cache"):
+        assert np.array_equal(getattr(e, name), getattr(c, name)), name
+    # and the rows really are the tokens the positions name
+    for s in range(B):
+        for h in range(H):
+            for j in range(int(c.fill[s, h])):
+                assert np.array_equal(a.k_cache[s, h, j], Kt[s, 2 + c.pos[s, h, j], h])

@@ -27,6 +27,12 @@ def test_noalloc_prefill_matches_ordinary_prefill_twice_in_a_row():
     for name in STATE:
         assert torch.equal(getattr(ref.gpu, name), getattr(new.gpu, name)), f"first call: {name}"
     assert int(ref.gpu.fill.min()) == 333
+    # the call itself takes no device memory: neither from the driver nor from torch's pool
+    torch.cuda.synchronize()
+    free_before, alloc_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+    new.gpu.prefill_compress_noalloc(new.dQ, new.dK, new.dV, new.dplen)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == alloc_before
     # second call right after it: shorter, ragged prompts (one below its budget), reversed token order as new data
     plen = torch.tensor([517, 120], dtype=torch.int32, device="cuda")
     q2, k2, v2 = (t.flip(2).contiguous() for t in (ref.dQ, ref.dK, ref.dV))
