@@ -66,6 +66,32 @@ def prefill_bytes_per_call(w, budgets, plens):
     return float(per_seq.sum()) * H
 
 
+NOMINAL_HBM_GBS = 8000.0  # the vendor's figure, for context beside the measured copy bandwidth
+RESOLVER_CYCLES_PER_STEP = 144.0  # one warp walking Algorithm 1's evicting steps in order (measured in isolation)
+
+
+def profiled_traffic(kernel, workload):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary profiles/<kernel>_<workload>.md (its line
+    'dram bytes per launch: N'), or None when there is no such summary."""
+    import re
+
+    path = os.path.join(ROOT, "profiles", f"{kernel}_{workload}.md")
+    if not os.path.exists(path):
+        return None, None
+    m = re.search(r"dram bytes per launch[^0-9]*([0-9][0-9_,]*)", open(path).read())
+    return (int(m.group(1).replace(",", "").replace("_", "")) if m else None), os.path.relpath(path, ROOT)
+
+
+def replay_bounds(w, budgets, plens, sms, sm_mhz):
+    """What bounds Section 3's sequential prompt replay in this design: every evicting step of a unit passes through
+    one resolver warp (a dependent chain of RESOLVER_CYCLES_PER_STEP cycles), one unit per SM at a time."""
+    N = plens.astype(np.int64)
+    C = np.minimum(budgets.astype(np.int64), N)
+    steps = float((N - C).sum()) * w.n_kv_heads  # evicting steps of one call, all units
+    clock = (sm_mhz or 1965.0) * 1e6
+    return steps, sms * clock / RESOLVER_CYCLES_PER_STEP  # steps per call, steps per second at the chain's pace
+
+
 # ------------------------------------------------------------------------------------------------- clocks
 
 class ClockSampler:
@@ -306,46 +332,194 @@ def run_ours(args, w):
     dec_gbs = dec_bytes * decode_calls / t_decode / 1e9
     pre_gbs = pre_bytes * R * K / t_prefill / 1e9
 
+    early = not args.no_early_inputs
+    decode_kernel = "decode_step_sm_kernel" if (early and units <= 4 * 148 and not args.packed_codes and d % 32 == 0) else "decode_step_kernel"
+    traffic, traffic_src = profiled_traffic(decode_kernel, w.name)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
         "ms_per_step": 1e3 * t_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u32", "data": "synthetic", "config": config_dict(w, R),
         "decode_us_per_call": 1e6 * t_decode / decode_calls,
         "decode_launch_mode": "cuda graph of he_decode_step calls" if graph is not None else "plain stream launches",
+        "decode_inputs": "HE_FLAG_EARLY_INPUTS: q, k, v of all steps are staged in HBM before the graph is launched, so each call "
+                         "may hash its rows under the previous call's scan" if early else "default order (rows read after the previous kernel ended)",
         "prefill_keys_per_s": prefill_rate, "prefill_ms_per_call": 1e3 * t_prefill / (R * K),
-        "roofline": {"kernel": "decode_step_kernel", "bound": "hbm", "achieved": dec_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": dec_gbs / peak, "peak_source": peak_src,
-                     "traffic": 10414848 if w.name == "throughput_batch" else None,
-                     "traffic_note": "dram read+write bytes of one launch from an ncu capture of this shape "
-                                     "(profiles/decode_step_kernel_throughput_batch.md): 10.4 MB read, the 4.8 MB "
-                                     "written are still in L2 when the kernel ends",
+        "roofline": {"kernel": decode_kernel, "bound": "hbm", "achieved": dec_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": dec_gbs / peak, "peak_source": peak_src, "frac_of_nominal_8TBs": dec_gbs / NOMINAL_HBM_GBS,
+                     "traffic": traffic, "traffic_source": traffic_src,
                      "algorithmic_bytes_per_launch": dec_bytes},
         "roofline_prefill": {"call": "he_prefill_compress (hash K, hash Q, replay, gather)", "bound": "hbm",
                              "achieved": pre_gbs, "peak": peak, "unit": "GB/s", "frac": pre_gbs / peak,
+                             "frac_of_nominal_8TBs": pre_gbs / NOMINAL_HBM_GBS,
                              "algorithmic_bytes_per_call": pre_bytes,
-                             "note": "the paper-exact replay is sequential per unit: bound by the step-to-step latency of its resolver warp and by tensor-core tile rate, not by HBM"},
+                             "note": "the HBM fraction of the whole call, as the metric asks; Section 3's replay phase is a "
+                                     "sequential dependent chain per unit, its own bound is in prefill_phases.replay_bound"},
         "gpu_launches": K * R * (6 + T),  # per prefill: W image, hash K, hash Q, schedule, replay, gather; per decode call: 1
         "input_setup_s": t_gen,
     }
 
+    from paper_2412_16187_b200 import prefill_phase_events
+
+    sms = torch.cuda.get_device_properties(local).multi_processor_count
+    sm_mhz = clocks.get("sm_mhz") if clocks else None
+
+    def phase_split(cache_list, dQ_, dK_, dV_, dplen_, Nmax_, ws_, reps=1):
+        """Milliseconds per call of the phases of he_prefill_compress, from events the library records around them
+        (the same kernels as in the timed region, one event record between two phases)."""
+        evs5 = [[ev() for _ in range(5)] for _ in range(len(cache_list) * reps)]
+        with torch.cuda.stream(stream):
+            k = 0
+            for _ in range(reps):
+                for c in cache_list:
+                    prefill_phase_events(evs5[k])
+                    c.prefill_compress(dQ_, dK_, dV_, dplen_, Nmax_, workspace=ws_, stream=stream)
+                    k += 1
+            prefill_phase_events(None)
+        torch.cuda.synchronize()
+        names = ("hash_k_ms", "hash_q_ms", "schedule_replay_ms", "gather_ms")
+        out = {n: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in evs5) for i, n in enumerate(names)}
+        out["call_ms"] = statistics.mean(e[0].elapsed_time(e[4]) for e in evs5)
+        return out
+
+    def replay_bound_obj(wk, budgets_, plens_, replay_ms):
+        steps, peak_steps = replay_bounds(wk, budgets_, plens_, sms, sm_mhz)
+        ach = steps / (replay_ms * 1e-3)
+        return {"bound": "latency: one resolver warp per SM walks a unit's evicting steps in order, a dependent chain of "
+                         f"{RESOLVER_CYCLES_PER_STEP:.0f} cycles per step", "unit": "evicting steps/s", "achieved": ach,
+                "peak": peak_steps, "frac": ach / peak_steps, "evicting_steps_per_call": steps,
+                "hbm_floor_ms_of_the_whole_call": None}
+
+    if rank == 0 and not args.skip_phases:
+        ph = phase_split(caches, dQ, dK, dV, dplen, Nmax, ws)
+        ph["replay_bound"] = replay_bound_obj(w, budgets, plens, ph["schedule_replay_ms"])
+        ph["replay_bound"]["hbm_floor_ms_of_the_whole_call"] = pre_bytes / (peak * 1e9) * 1e3
+        line["prefill_phases"] = ph
+
+    T2 = min(T, args.secondary_steps)
+
+    def timed_decode_graph(steps_):
+        """us per call of `steps_` decode steps x R replicas captured into a CUDA graph with the caches' current config."""
+        with torch.cuda.stream(stream):
+            stream.synchronize()
+            g2 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g2, stream=stream):
+                for i in range(steps_):
+                    for r, c in enumerate(caches):
+                        c.decode_step(gq[i], gk[i], gv[i], victim_out=victims[r], stream=stream)
+            g2.replay()
+            a0, a1 = ev(), ev()
+            a0.record(stream)
+            g2.replay()
+            g2.replay()
+            a1.record(stream)
+        torch.cuda.synchronize()
+        return a0.elapsed_time(a1) * 1e3 / (2 * steps_ * R)
+
+    if rank == 0 and not args.skip_decode_variants:
+        from paper_2412_16187_b200 import HE_FLAG_EARLY_INPUTS, lib as he_lib
+        import ctypes
+
+        dv = {}
+        # (a) the default order: q, k, v read only after the stream's previous kernel has ended
+        for c in caches:
+            c.cfg.flags &= ~HE_FLAG_EARLY_INPUTS
+        us = timed_decode_graph(T2)
+        dv["default_order"] = {"us_per_call": us, "frac": dec_bytes / us / 1e3 / peak,
+                               "what": "HE_FLAG_EARLY_INPUTS off: the rows may come from the kernel enqueued just before the call"}
+        for c in caches:
+            c.cfg.flags |= HE_FLAG_EARLY_INPUTS if early else 0
+        # (b) plain stream launches instead of a graph: the host enqueues every call (ctypes, addresses looked up once)
+        L = he_lib()
+        ptrs = [(ctypes.byref(c.cfg), ctypes.byref(c.ca), victims[r].data_ptr()) for r, c in enumerate(caches)]
+        ins = [(gq[i].data_ptr(), gk[i].data_ptr(), gv[i].data_ptr()) for i in range(T2)]
+        sp = stream.cuda_stream
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            for rep_ in range(2):
+                if rep_ == 1:
+                    torch.cuda.synchronize()
+                    a0, a1 = ev(), ev()
+                    t0 = time.perf_counter()
+                    a0.record(stream)
+                for q_, k_, v_ in ins:
+                    for cf, ca_, vp_ in ptrs:
+                        L.he_decode_step(cf, ca_, q_, k_, v_, vp_, None, None, sp)
+            a1.record(stream)
+            t_host = time.perf_counter() - t0
+        torch.cuda.synchronize()
+        dv["plain_launch"] = {"us_per_call": a0.elapsed_time(a1) * 1e3 / (T2 * R), "host_enqueue_us_per_call": 1e6 * t_host / (T2 * R),
+                              "what": "the same calls as plain stream launches, enqueued one by one from the host"}
+        # (c) one replica only: its 15 MB of tables, scores and slots stay in L2 between steps
+        c0 = caches[0]
+        with torch.cuda.stream(stream):
+            stream.synchronize()
+            g1 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g1, stream=stream):
+                for i in range(T2):
+                    c0.decode_step(gq[i], gk[i], gv[i], victim_out=victims[0], stream=stream)
+            g1.replay()
+            a0, a1 = ev(), ev()
+            a0.record(stream)
+            g1.replay()
+            g1.replay()
+            a1.record(stream)
+        torch.cuda.synchronize()
+        us = a0.elapsed_time(a1) * 1e3 / (2 * T2)
+        dv["single_replica_l2_warm"] = {"us_per_call": us, "frac_of_hbm_peak": dec_bytes / us / 1e3 / peak,
+                                        "what": "one cache stepped again and again: its working set stays in L2, so this is not an HBM figure"}
+        line["decode_variants"] = dv
+        del g1
+
+    if rank == 0 and not args.skip_protected and w.n_sink == 0 and w.n_recent == 0:
+        # ---- the paper's own setting (Section 4, configuration and setup): the first 4 and the newest 10 tokens stay
+        for c in caches:
+            c.cfg.n_sink, c.cfg.n_recent = 4, 10
+        with torch.cuda.stream(stream):
+            prefill_all()
+            p0, p1 = ev(), ev()
+            p0.record(stream)
+            prefill_all()
+            p1.record(stream)
+        torch.cuda.synchronize()
+        us = timed_decode_graph(T2)
+        line["protected_4_10"] = {"n_sink": 4, "n_recent": 10, "prefill_ms_per_call": p0.elapsed_time(p1) / R,
+                                  "decode_us_per_call": us, "decode_frac": dec_bytes / us / 1e3 / peak}
+        for c in caches:
+            c.cfg.n_sink, c.cfg.n_recent = 0, 0
+        with torch.cuda.stream(stream):
+            prefill_all()
+        torch.cuda.synchronize()
+
     if rank == 0 and not args.skip_e2e:
-        # ---- end to end: host buffers in, victims out, through he_decode_step_host (copies inside the timed region)
+        # ---- end to end: host buffers in, victims out, through he_decode_step_host_enqueue (copies inside the timed
+        # region). Each step's q, k, v sit in one pinned block at the offsets the call recognises (one copy in), the
+        # victims come back in one copy; addresses are looked up once, as a serving loop would.
         n_e2e = min(T, args.e2e_steps)
-        hq, hk, hv = (x[:n_e2e].cpu().pin_memory() for x in (gq, gk, gv))
+        esz = gq.element_size()
+        qb, kb = gq[0].numel() * esz, gk[0].numel() * esz
+        al = lambda x: (x + 255) // 256 * 256
+        blk = al(qb) + al(kb) + al(kb)
+        hblock = torch.empty((n_e2e, blk), dtype=torch.uint8).pin_memory()
+        for i in range(n_e2e):
+            hblock[i, :qb] = gq[i].contiguous().view(torch.uint8).flatten().cpu()
+            hblock[i, al(qb):al(qb) + kb] = gk[i].contiguous().view(torch.uint8).flatten().cpu()
+            hblock[i, al(qb) + al(kb):al(qb) + al(kb) + kb] = gv[i].contiguous().view(torch.uint8).flatten().cpu()
         # The layer replicas' calls of a step are independent, so they alternate between two streams (each with its
-        # own staging): the host->device copies of one overlap the kernel of the other. Every step ends with a
-        # synchronise, after which that step's victims are readable on the host.
+        # own staging): the copies of one overlap the kernel of the other. Every step ends with a synchronise, after
+        # which that step's victims are readable on the host.
         hvic = torch.empty((R, B, H), dtype=torch.int32).pin_memory()
         e_streams = [torch.cuda.Stream(), torch.cuda.Stream()]
         stagings = [torch.empty(decode_staging_bytes(caches[0].cfg), dtype=torch.uint8, device="cuda") for _ in e_streams]
-
-        rows = [(hq[i], hk[i], hv[i]) for i in range(n_e2e)]  # views of the pinned buffers, one per step
-        outs = [hvic[r] for r in range(R)]
+        base = hblock.data_ptr()
+        calls = [(c, hvic[r].data_ptr(), stagings[r & 1].data_ptr(), stagings[r & 1].numel(), e_streams[r & 1].cuda_stream)
+                 for r, c in enumerate(caches)]
 
         def e2e_step(i):
-            q_i, k_i, v_i = rows[i]
-            for r, c in enumerate(caches):
-                c.decode_step_host_enqueue(q_i, k_i, v_i, outs[r], stagings[r & 1], stream=e_streams[r & 1])
+            qp = base + i * blk
+            kp = qp + al(qb)
+            vp = kp + al(kb)
+            for c, op, sp_, sn, st_ in calls:
+                c.decode_step_host_enqueue_raw(qp, kp, vp, op, sp_, sn, st_)
             for s_ in e_streams:
                 s_.synchronize()
             return int(hvic[R - 1, 0, 0])  # the step's result is read on the host
@@ -357,12 +531,11 @@ def run_ours(args, w):
         for i in range(n_e2e):
             e2e_step(i)
         t_e2e = time.perf_counter() - t0
-        h2d = (hq[0].numel() + hk[0].numel() + hv[0].numel()) * hq.element_size()
-        line["e2e"] = {"value": units * n_e2e * R * world / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                       "d2h_bytes_per_step": hvic[0].numel() * 4,
+        line["e2e"] = {"value": units * n_e2e * R * world / t_e2e, "unit": UNIT, "h2d_bytes_per_step": qb + 2 * kb,
+                       "d2h_bytes_per_step": hvic[0].numel() * 4, "us_per_call": 1e6 * t_e2e / (n_e2e * R),
                        "what": f"he_decode_step_host_enqueue, {n_e2e} decode steps x {R} layer replicas on two alternating streams, "
-                               "one synchronise and one host read of the victims per step; pinned host q/k/v copied in and "
-                               "victims copied out by every call inside the timed region"}
+                               "one synchronise and one host read of the victims per step; every call copies its pinned host "
+                               "q/k/v block in (one copy) and its victims out inside the timed region"}
 
     if rank == 0 and not args.skip_folded and R > 1:
         # ---- secondary figure: the same decode kernel with all R replicas folded into ONE call (batch R*B), i.e. when
@@ -474,6 +647,39 @@ def run_ours(args, w):
                                   "mean_loss": losses, "ms_per_call": ms, "achieved_gbs": lbytes / (ms * 1e-3) / 1e9,
                                   "frac": lbytes / (ms * 1e-3) / 1e9 / peak}
 
+    if rank == 0 and not args.skip_largest_prefill and w.name == "throughput_batch":
+        # ---- he_prefill_compress on the configuration that is largest for prefill: long_prefill, its 32 layers folded
+        # into the batch (256 units, 32768-token prompts, 9830 slots). Layer 0's q/k/v are generated on the host by the
+        # seeded generator; the other 31 layers are that layer's tokens rotated by a layer-dependent offset on the
+        # device (same distribution, different order, own memory: 12.9 GB), which keeps the set-up to seconds.
+        w4 = wl.CONFIGS["long_prefill"]
+        B4, N4 = w4.n_seq, w4.max_prompt_len
+        k0, v0, q0 = (up(wl.gen_tokens(w4, x, 0, 1, 0, N4)[0]) for x in "kvq")
+        dK4 = torch.empty((B4, H, N4, d), dtype=tdt, device="cuda")
+        dV4 = torch.empty_like(dK4)
+        dQ4 = torch.empty((B4, w4.n_kv_heads * w4.group_size, N4, d), dtype=tdt, device="cuda")
+        for l in range(B4):
+            dK4[l], dV4[l], dQ4[l] = (torch.roll(x, shifts=l * 997, dims=1) for x in (k0, v0, q0))
+        b4, p4 = w4.budgets(), w4.prompt_lens()
+        c4 = HashEvictCache(B4, w4.n_kv_heads, w4.group_size, d, w4.hash_bits, b4, torch.from_numpy(wl.gen_W(w4)), dtype=tdt)
+        ws4 = c4.workspace(N4)
+        dp4 = torch.from_numpy(p4).cuda()
+        with torch.cuda.stream(stream):
+            c4.prefill_compress(dQ4, dK4, dV4, dp4, N4, workspace=ws4, stream=stream)
+        torch.cuda.synchronize()
+        ph4 = phase_split([c4], dQ4, dK4, dV4, dp4, N4, ws4, reps=3)
+        bytes4 = prefill_bytes_per_call(w4, b4, p4)
+        ph4["replay_bound"] = replay_bound_obj(w4, b4, p4, ph4["schedule_replay_ms"])
+        ph4["replay_bound"]["hbm_floor_ms_of_the_whole_call"] = bytes4 / (peak * 1e9) * 1e3
+        gbs4 = bytes4 / (ph4["call_ms"] * 1e-3) / 1e9
+        line["prefill_largest"] = {"workload": "long_prefill, 32 layers folded into the batch (256 units, N = 32768, C = 9830)",
+                                   "ms_per_call": ph4["call_ms"], "keys_per_s": float(p4.sum()) * w4.n_kv_heads / (ph4["call_ms"] * 1e-3),
+                                   "bound": "hbm", "achieved": gbs4, "peak": peak, "unit": "GB/s", "frac": gbs4 / peak,
+                                   "frac_of_nominal_8TBs": gbs4 / NOMINAL_HBM_GBS, "algorithmic_bytes_per_call": bytes4,
+                                   "phases": ph4,
+                                   "data": "layer 0 from the seeded generator, layers 1..31 = layer 0 with its tokens rotated by 997 * layer"}
+        del dK4, dV4, dQ4, c4, ws4, k0, v0, q0
+
     if rank == 0:
         line["clocks"] = clocks
         if not args.skip_cpu_baseline and world == 1:
@@ -482,6 +688,9 @@ def run_ours(args, w):
             line["cpu_baseline"] = {"value": r["evictions_per_s"], "unit": UNIT, "cores": threads, "kind": "oracle",
                                     "sample": r["sample"], "prefill_keys_per_s": r["prefill_keys_per_s"],
                                     "seconds": r["t_prefill_s"] + r["t_decode_s"]}
+            r1 = oracle_sample(w, 1, min(32, args.ref_decode_steps), 1)
+            line["cpu_baseline"].update(value_1_thread=r1["evictions_per_s"], prefill_keys_per_s_1_thread=r1["prefill_keys_per_s"],
+                                        sample_1_thread=r1["sample"], seconds_1_thread=r1["t_prefill_s"] + r1["t_decode_s"])
         line["wall_s_timed_region"] = t_wall
         print(json.dumps(line))
     if world > 1:
@@ -506,6 +715,11 @@ def main():
     ap.add_argument("--no-early-inputs", action="store_true",
                     help="leave HE_FLAG_EARLY_INPUTS off (q, k, v are then read only after the stream's previous kernel has ended)")
     ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-phases", action="store_true", help="skip the per-phase split of he_prefill_compress")
+    ap.add_argument("--skip-decode-variants", action="store_true", help="skip default-order / plain-launch / one-replica decode figures")
+    ap.add_argument("--skip-protected", action="store_true", help="skip the figures with the paper's protected windows (4, 10)")
+    ap.add_argument("--skip-largest-prefill", action="store_true", help="skip he_prefill_compress on long_prefill (32 layers folded)")
+    ap.add_argument("--secondary-steps", type=int, default=128, help="decode steps of the secondary decode figures")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-oneshot", action="store_true", help="skip the he_prefill_oneshot figure")
     ap.add_argument("--skip-attend", action="store_true", help="skip the he_attend figure")

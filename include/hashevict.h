@@ -187,7 +187,9 @@ int he_reset(const he_config* cfg, const he_cache* cache, void* stream);
  *     caller can keep several streams busy (say, the caches of different layers on alternating streams, each with
  *     its own staging, copies of one overlapping the kernel of the other). victim_host holds the result, and
  *     q/k/v_host and staging may be reused, only once `stream` has been synchronised; the host buffers must be
- *     pinned for the copies to be asynchronous.
+ *     pinned for the copies to be asynchronous. When the three host tensors lie in one block - k_host = q_host +
+ *     round_up(bytes of q, 256), v_host = k_host + round_up(bytes of k, 256) - they travel in a single copy (three
+ *     driver calls per step instead of five; at under 1 MB per step the calls, not the bus, set the pace).
  *   he_prefill_compress_host: q [B, Hkv*G, Nmax, d], k, v [B, Hkv, Nmax, d] contiguous host tensors,
  *     prompt_len_host [B]; fill_host [B, Hkv] receives the valid-slot counts. staging: >=
  *     he_prefill_staging_bytes(cfg, max_prompt_len) device bytes (includes the prompt-code workspace).
@@ -298,6 +300,16 @@ int he_prefill_compress_noalloc(const he_config* cfg, const he_cache* cache, con
  * Diagnostic only: the paper has no counterpart.
  */
 int he_device_error_count(void);
+
+/*
+ * he_prefill_phase_events - timing aid (the paper has no counterpart). events: five cudaEvent_t handles (as void*)
+ * created by the caller with timing enabled, or NULL to switch the aid off. While set, every prefill call of the
+ * calling thread (he_prefill_compress and its variants) records them on its stream around its phases, launching
+ * exactly the kernels it always launches: [0] start, [1] after Eq. 2 on the prompt keys (with the W image), [2] after
+ * Eq. 2 on the queries, [3] after the unit schedule and the replay (or ranking), [4] after the K / V gather. An event
+ * record is one more stream operation between two kernels, so use it for measurement runs only.
+ */
+int he_prefill_phase_events(void* const* events);
 
 /* Text of the calling thread's most recent error ("" if none). The pointer stays valid until the next failing call. */
 const char* he_last_error(void);

@@ -38,7 +38,7 @@ class he_cache(ctypes.Structure):
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
     "he_decode_staging_bytes", "he_decode_step_host", "he_decode_step_host_enqueue", "he_prefill_staging_bytes", "he_prefill_compress_host",
-    "he_prefill_compress_noalloc", "he_attend", "he_prefill_oneshot", "he_oneshot_workspace_bytes", "he_prefill_oneshot_l2", "he_attention_loss", "he_decode_step_l2", "he_step_scratch_bytes", "he_device_error_count", "he_last_error",
+    "he_prefill_compress_noalloc", "he_attend", "he_prefill_oneshot", "he_oneshot_workspace_bytes", "he_prefill_oneshot_l2", "he_attention_loss", "he_decode_step_l2", "he_step_scratch_bytes", "he_device_error_count", "he_prefill_phase_events", "he_last_error",
 )
 
 _lib = None
@@ -83,6 +83,8 @@ def lib():
     L.he_attend.restype = ctypes.c_int
     L.he_step_scratch_bytes.argtypes = [cfgp]
     L.he_step_scratch_bytes.restype = sz
+    L.he_prefill_phase_events.argtypes = [ctypes.POINTER(vp)]
+    L.he_prefill_phase_events.restype = ctypes.c_int
     L.he_device_error_count.argtypes = []
     L.he_device_error_count.restype = ctypes.c_int
     L.he_last_error.argtypes = []
@@ -97,6 +99,19 @@ def lib():
 def device_error_count() -> int:
     """he_device_error_count: thread blocks that gave up on a bounded wait (0 in a healthy process). Synchronises."""
     return lib().he_device_error_count()
+
+
+def prefill_phase_events(events=None):
+    """he_prefill_phase_events: five torch.cuda.Event(enable_timing=True) that the next prefill calls of this thread
+    record around their phases (hash K, hash Q, schedule + replay, gather), or None to switch that off."""
+    if events is None:
+        lib().he_prefill_phase_events(None)
+        return
+    assert len(events) == 5
+    for e in events:
+        e.record()  # torch creates the underlying cudaEvent lazily, on first record
+    arr = (ctypes.c_void_p * 5)(*[e.cuda_event for e in events])
+    lib().he_prefill_phase_events(arr)
 
 
 def _check(rc: int):
@@ -300,6 +315,12 @@ class HashEvictCache:
         """he_decode_step_host_enqueue: as decode_step_host but without the final synchronise (results after a stream sync)."""
         _check(lib().he_decode_step_host_enqueue(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q_host), _ptr(k_host),
                                                  _ptr(v_host), _ptr(victim_host), _ptr(staging), staging.numel(), _stream(stream)))
+
+    def decode_step_host_enqueue_raw(self, q_ptr, k_ptr, v_ptr, victim_ptr, staging_ptr, staging_bytes, stream_ptr):
+        """he_decode_step_host_enqueue on addresses the caller has already looked up (a serving loop reuses its pinned
+        buffers, so it need not ask torch for data_ptr() and the stream handle at every step)."""
+        _check(lib().he_decode_step_host_enqueue(ctypes.byref(self.cfg), ctypes.byref(self.ca), q_ptr, k_ptr, v_ptr, victim_ptr,
+                                                 staging_ptr, staging_bytes, stream_ptr))
 
     def prefill_compress_host(self, q_host, k_host, v_host, prompt_len_host, max_prompt_len, fill_host, staging, stream=None):
         _check(lib().he_prefill_compress_host(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q_host), _ptr(k_host),

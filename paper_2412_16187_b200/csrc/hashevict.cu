@@ -40,6 +40,12 @@ using namespace he;
 namespace {
 
 thread_local char g_err[512] = "";
+thread_local cudaEvent_t g_phase_events[5] = {};  // he_prefill_phase_events: recorded between the phases of a prefill call
+thread_local bool g_phase_events_on = false;
+
+void record_phase(int i, cudaStream_t st) {
+  if (g_phase_events_on && g_phase_events[i] != nullptr) cudaEventRecord(g_phase_events[i], st);
+}
 
 int fail(int code, const char* fmt, ...) {
   va_list ap;
@@ -514,6 +520,12 @@ extern "C" {
 
 const char* he_last_error(void) { return g_err; }
 
+int he_prefill_phase_events(void* const* events) {
+  g_phase_events_on = events != nullptr;
+  for (int i = 0; i < 5; ++i) g_phase_events[i] = events != nullptr ? static_cast<cudaEvent_t>(events[i]) : nullptr;
+  return HE_OK;
+}
+
 int he_device_error_count(void) {
   int n = 0;
   if (cudaMemcpyFromSymbol(&n, he::g_tc_error, sizeof(int)) != cudaSuccess) return -1;
@@ -682,6 +694,7 @@ int prefill_impl(int variant /* 0: Algorithm 1, 1: averaged Hamming, 2: L2 norm 
                                                  align_up((size_t)units * max_prompt_len * Wd * 4, 256));
 
   bool image_built = false;
+  record_phase(0, st);
   // phase 1: Eq. 2 on every prompt key and on the queries of the tokens that will evict
   HashJob job{};
   job.w_image = static_cast<char*>(workspace) + align_up((size_t)units * max_prompt_len * Wd * 4, 256) +
@@ -703,6 +716,7 @@ int prefill_impl(int variant /* 0: Algorithm 1, 1: averaged Hamming, 2: L2 norm 
   job.s1 = kv_strides[1];
   job.s2 = kv_strides[2];
   if (int rc = launch_hash(job, max_prompt_len, (int)units, st, &image_built)) return rc;
+  record_phase(1, st);
   if (variant != 2) {
   job.x = q;
   job.out = qcodes;
@@ -715,6 +729,7 @@ int prefill_impl(int variant /* 0: Algorithm 1, 1: averaged Hamming, 2: L2 norm 
   if (int rc = launch_hash(job, max_prompt_len, (int)units * G, st, &image_built)) return rc;
   }
 
+  record_phase(2, st);
   // phase 2: the sequential replay of Algorithm 1 over the prompt, one CTA per unit
   int32_t* sched = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(qcodes) +
                                               align_up((size_t)units * max_prompt_len * G * Wd * 4, 256));
@@ -742,6 +757,7 @@ int prefill_impl(int variant /* 0: Algorithm 1, 1: averaged Hamming, 2: L2 norm 
     if (int rc = (Wd == 1 ? launch_replay<1>(ra, units, st) : launch_replay<2>(ra, units, st))) return rc;
   }
 
+  record_phase(3, st);
   // phase 3: surviving K / V rows into their slots
   GatherArgs ga{*cfg, *cache, k, v, kv_strides[0], kv_strides[1], kv_strides[2], max_prompt_len};
   const long long per_unit = 2LL * cfg->max_budget * (cfg->head_dim * es / 16);
@@ -749,6 +765,7 @@ int prefill_impl(int variant /* 0: Algorithm 1, 1: averaged Hamming, 2: L2 norm 
   if (units > 65535) return fail(HE_ERR_UNSUPPORTED, "more than 65535 units in one prefill call");
   prefill_gather_kernel<<<dim3((unsigned)gx, (unsigned)units), kGatherThreads, 0, st>>>(ga);
   HE_CUDA_CHECK(cudaGetLastError());
+  record_phase(4, st);
   return HE_OK;
 }
 
@@ -936,9 +953,19 @@ int he_decode_step_host_enqueue(const he_config* cfg, const he_cache* cache, con
   void* dv = p;
   p += align_up(units * row, 256);
   int32_t* dvictim = reinterpret_cast<int32_t*>(p);
-  HE_CUDA_CHECK(cudaMemcpyAsync(dq, q_host, units * cfg->group_size * row, cudaMemcpyHostToDevice, st));
-  HE_CUDA_CHECK(cudaMemcpyAsync(dk, k_host, units * row, cudaMemcpyHostToDevice, st));
-  HE_CUDA_CHECK(cudaMemcpyAsync(dv, v_host, units * row, cudaMemcpyHostToDevice, st));
+  // One copy when the three host tensors already sit in one block at the staging area's own offsets (q, then k,
+  // then v, each starting on the next 256-byte boundary): every driver call costs the host a few microseconds, and
+  // at these sizes (under 1 MB per step) that, not the bus, is what an end-to-end step pays for.
+  const size_t qb = units * cfg->group_size * row, kb = units * row;
+  const char* hq = static_cast<const char*>(q_host);
+  if (static_cast<const char*>(k_host) == hq + align_up(qb, 256) &&
+      static_cast<const char*>(v_host) == hq + align_up(qb, 256) + align_up(kb, 256)) {
+    HE_CUDA_CHECK(cudaMemcpyAsync(dq, q_host, align_up(qb, 256) + align_up(kb, 256) + kb, cudaMemcpyHostToDevice, st));
+  } else {
+    HE_CUDA_CHECK(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st));
+    HE_CUDA_CHECK(cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, st));
+    HE_CUDA_CHECK(cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, st));
+  }
   if (int rc = he_decode_step(cfg, cache, dq, dk, dv, dvictim, nullptr, nullptr, stream)) return rc;
   HE_CUDA_CHECK(cudaMemcpyAsync(victim_host, dvictim, units * 4, cudaMemcpyDeviceToHost, st));
   return HE_OK;
