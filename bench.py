@@ -497,13 +497,13 @@ def run_ours(args, w):
         n_e2e = min(T, args.e2e_steps)
         esz = gq.element_size()
         qb, kb = gq[0].numel() * esz, gk[0].numel() * esz
-        al = lambda x: (x + 255) // 256 * 256
-        blk = al(qb) + al(kb) + al(kb)
+        blk_bytes, (oq, ok_, ov) = caches[0].host_block_layout()
+        blk = (blk_bytes + 255) // 256 * 256
         hblock = torch.empty((n_e2e, blk), dtype=torch.uint8).pin_memory()
         for i in range(n_e2e):
-            hblock[i, :qb] = gq[i].contiguous().view(torch.uint8).flatten().cpu()
-            hblock[i, al(qb):al(qb) + kb] = gk[i].contiguous().view(torch.uint8).flatten().cpu()
-            hblock[i, al(qb) + al(kb):al(qb) + al(kb) + kb] = gv[i].contiguous().view(torch.uint8).flatten().cpu()
+            hblock[i, oq:oq + qb] = gq[i].contiguous().view(torch.uint8).flatten().cpu()
+            hblock[i, ok_:ok_ + kb] = gk[i].contiguous().view(torch.uint8).flatten().cpu()
+            hblock[i, ov:ov + kb] = gv[i].contiguous().view(torch.uint8).flatten().cpu()
         # The layer replicas' calls of a step are independent, so they alternate between two streams (each with its
         # own staging): the copies of one overlap the kernel of the other. Every step ends with a synchronise, after
         # which that step's victims are readable on the host.
@@ -516,10 +516,8 @@ def run_ours(args, w):
 
         def e2e_step(i):
             qp = base + i * blk
-            kp = qp + al(qb)
-            vp = kp + al(kb)
             for c, op, sp_, sn, st_ in calls:
-                c.decode_step_host_enqueue_raw(qp, kp, vp, op, sp_, sn, st_)
+                c.decode_step_host_block_enqueue_raw(qp, op, sp_, sn, st_)
             for s_ in e_streams:
                 s_.synchronize()
             return int(hvic[R - 1, 0, 0])  # the step's result is read on the host
@@ -533,7 +531,7 @@ def run_ours(args, w):
         t_e2e = time.perf_counter() - t0
         line["e2e"] = {"value": units * n_e2e * R * world / t_e2e, "unit": UNIT, "h2d_bytes_per_step": qb + 2 * kb,
                        "d2h_bytes_per_step": hvic[0].numel() * 4, "us_per_call": 1e6 * t_e2e / (n_e2e * R),
-                       "what": f"he_decode_step_host_enqueue, {n_e2e} decode steps x {R} layer replicas on two alternating streams, "
+                       "what": f"he_decode_step_host_block_enqueue, {n_e2e} decode steps x {R} layer replicas on two alternating streams, "
                                "one synchronise and one host read of the victims per step; every call copies its pinned host "
                                "q/k/v block in (one copy) and its victims out inside the timed region"}
 

@@ -187,9 +187,11 @@ int he_reset(const he_config* cfg, const he_cache* cache, void* stream);
  *     caller can keep several streams busy (say, the caches of different layers on alternating streams, each with
  *     its own staging, copies of one overlapping the kernel of the other). victim_host holds the result, and
  *     q/k/v_host and staging may be reused, only once `stream` has been synchronised; the host buffers must be
- *     pinned for the copies to be asynchronous. When the three host tensors lie in one block - k_host = q_host +
- *     round_up(bytes of q, 256), v_host = k_host + round_up(bytes of k, 256) - they travel in a single copy (three
- *     driver calls per step instead of five; at under 1 MB per step the calls, not the bus, set the pace).
+ *     pinned for the copies to be asynchronous.
+ *   he_decode_step_host_block_enqueue: the same with q, k, v in ONE host block (one pinned allocation), q at offset 0,
+ *     k and v at the offsets he_decode_host_block_bytes reports (each tensor starts on the next 256-byte boundary; the
+ *     function returns the block's size). The block travels in a single copy: three driver calls per step instead of
+ *     five, which matters because at under 1 MB per step the calls cost the host more than the bus costs the copy.
  *   he_prefill_compress_host: q [B, Hkv*G, Nmax, d], k, v [B, Hkv, Nmax, d] contiguous host tensors,
  *     prompt_len_host [B]; fill_host [B, Hkv] receives the valid-slot counts. staging: >=
  *     he_prefill_staging_bytes(cfg, max_prompt_len) device bytes (includes the prompt-code workspace).
@@ -199,6 +201,9 @@ int he_decode_step_host(const he_config* cfg, const he_cache* cache, const void*
                         const void* v_host, int32_t* victim_host, void* staging, size_t staging_bytes, void* stream);
 int he_decode_step_host_enqueue(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
                                 const void* v_host, int32_t* victim_host, void* staging, size_t staging_bytes, void* stream);
+size_t he_decode_host_block_bytes(const he_config* cfg, size_t offsets[3]);
+int he_decode_step_host_block_enqueue(const he_config* cfg, const he_cache* cache, const void* qkv_host, int32_t* victim_host,
+                                      void* staging, size_t staging_bytes, void* stream);
 size_t he_prefill_staging_bytes(const he_config* cfg, int32_t max_prompt_len);
 int he_prefill_compress_host(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
                              const void* v_host, const int32_t* prompt_len_host, int32_t max_prompt_len,

@@ -37,7 +37,7 @@ class he_cache(ctypes.Structure):
 
 EXPORTS = (
     "he_hash_keys", "he_decode_step", "he_prefill_compress", "he_workspace_bytes", "he_reset",
-    "he_decode_staging_bytes", "he_decode_step_host", "he_decode_step_host_enqueue", "he_prefill_staging_bytes", "he_prefill_compress_host",
+    "he_decode_staging_bytes", "he_decode_step_host", "he_decode_step_host_enqueue", "he_decode_step_host_block_enqueue", "he_decode_host_block_bytes", "he_prefill_staging_bytes", "he_prefill_compress_host",
     "he_prefill_compress_noalloc", "he_attend", "he_prefill_oneshot", "he_oneshot_workspace_bytes", "he_prefill_oneshot_l2", "he_attention_loss", "he_decode_step_l2", "he_step_scratch_bytes", "he_device_error_count", "he_prefill_phase_events", "he_last_error",
 )
 
@@ -69,6 +69,10 @@ def lib():
     L.he_decode_staging_bytes.restype = sz
     L.he_decode_step_host.argtypes = [cfgp, cap, vp, vp, vp, vp, vp, sz, vp]
     L.he_decode_step_host_enqueue.argtypes = [cfgp, cap, vp, vp, vp, vp, vp, sz, vp]
+    L.he_decode_step_host_block_enqueue.argtypes = [cfgp, cap, vp, vp, vp, sz, vp]
+    L.he_decode_step_host_block_enqueue.restype = ctypes.c_int
+    L.he_decode_host_block_bytes.argtypes = [cfgp, ctypes.POINTER(sz)]
+    L.he_decode_host_block_bytes.restype = sz
     L.he_prefill_staging_bytes.argtypes = [cfgp, i32]
     L.he_prefill_staging_bytes.restype = sz
     L.he_prefill_compress_host.argtypes = [cfgp, cap, vp, vp, vp, vp, i32, vp, vp, sz, vp]
@@ -316,11 +320,17 @@ class HashEvictCache:
         _check(lib().he_decode_step_host_enqueue(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q_host), _ptr(k_host),
                                                  _ptr(v_host), _ptr(victim_host), _ptr(staging), staging.numel(), _stream(stream)))
 
-    def decode_step_host_enqueue_raw(self, q_ptr, k_ptr, v_ptr, victim_ptr, staging_ptr, staging_bytes, stream_ptr):
-        """he_decode_step_host_enqueue on addresses the caller has already looked up (a serving loop reuses its pinned
-        buffers, so it need not ask torch for data_ptr() and the stream handle at every step)."""
-        _check(lib().he_decode_step_host_enqueue(ctypes.byref(self.cfg), ctypes.byref(self.ca), q_ptr, k_ptr, v_ptr, victim_ptr,
-                                                 staging_ptr, staging_bytes, stream_ptr))
+    def host_block_layout(self):
+        """he_decode_host_block_bytes: (bytes of the one-block host layout of a step's q, k, v; their three offsets)."""
+        offs = (ctypes.c_size_t * 3)()
+        n = lib().he_decode_host_block_bytes(ctypes.byref(self.cfg), offs)
+        return n, tuple(offs)
+
+    def decode_step_host_block_enqueue_raw(self, qkv_ptr, victim_ptr, staging_ptr, staging_bytes, stream_ptr):
+        """he_decode_step_host_block_enqueue on addresses the caller has already looked up (a serving loop reuses its
+        pinned buffers, so it need not ask torch for data_ptr() and the stream handle at every step)."""
+        _check(lib().he_decode_step_host_block_enqueue(ctypes.byref(self.cfg), ctypes.byref(self.ca), qkv_ptr, victim_ptr,
+                                                       staging_ptr, staging_bytes, stream_ptr))
 
     def prefill_compress_host(self, q_host, k_host, v_host, prompt_len_host, max_prompt_len, fill_host, staging, stream=None):
         _check(lib().he_prefill_compress_host(ctypes.byref(self.cfg), ctypes.byref(self.ca), _ptr(q_host), _ptr(k_host),

@@ -173,7 +173,7 @@ __global__ void __launch_bounds__(kSmThreads, 2) decode_step_sm_kernel(const Dec
   __syncthreads();
   const he_config& cfg = cfg_s;
   const int d = cfg.head_dim, b = cfg.hash_bits, G = cfg.group_size, es = esize_of(cfg.dtype);
-  const int Cmax = cfg.max_budget, H = cfg.n_kv_heads;
+  const int Cmax = cfg.max_budget;
   const int R = G + 1;
   const int cpr = d * es / 16;  // 16-byte chunks per row
   const void* const q_in = in_s[0];

@@ -938,7 +938,8 @@ int he_decode_step_host(const he_config* cfg, const he_cache* cache, const void*
 int he_decode_step_host_enqueue(const he_config* cfg, const he_cache* cache, const void* q_host, const void* k_host,
                                 const void* v_host, int32_t* victim_host, void* staging, size_t staging_bytes, void* stream) {
   if (int rc = check_config(cfg, true)) return rc;
-  if (!q_host || !k_host || !v_host || !victim_host || !staging) return fail(HE_ERR_INVALID_ARG, "a host pointer or staging is null");
+  const bool block = q_host != nullptr && k_host == nullptr && v_host == nullptr;  // the one-block form (internal)
+  if (!q_host || (!block && (!k_host || !v_host)) || !victim_host || !staging) return fail(HE_ERR_INVALID_ARG, "a host pointer or staging is null");
   if ((reinterpret_cast<uintptr_t>(staging) & 255u) != 0) return fail(HE_ERR_INVALID_ARG, "staging must be 256-byte aligned");
   const size_t need = he_decode_staging_bytes(cfg);
   if (staging_bytes < need) return fail(HE_ERR_WORKSPACE, "staging has %zu bytes, %zu needed", staging_bytes, need);
@@ -953,13 +954,11 @@ int he_decode_step_host_enqueue(const he_config* cfg, const he_cache* cache, con
   void* dv = p;
   p += align_up(units * row, 256);
   int32_t* dvictim = reinterpret_cast<int32_t*>(p);
-  // One copy when the three host tensors already sit in one block at the staging area's own offsets (q, then k,
-  // then v, each starting on the next 256-byte boundary): every driver call costs the host a few microseconds, and
-  // at these sizes (under 1 MB per step) that, not the bus, is what an end-to-end step pays for.
   const size_t qb = units * cfg->group_size * row, kb = units * row;
-  const char* hq = static_cast<const char*>(q_host);
-  if (static_cast<const char*>(k_host) == hq + align_up(qb, 256) &&
-      static_cast<const char*>(v_host) == hq + align_up(qb, 256) + align_up(kb, 256)) {
+  if (k_host == nullptr && v_host == nullptr) {
+    // he_decode_step_host_block_enqueue: q, k, v in one host block laid out like the staging area, one copy. Every
+    // driver call costs the host a few microseconds, and at these sizes (under 1 MB per step) that, not the bus, is
+    // what an end-to-end step pays for first.
     HE_CUDA_CHECK(cudaMemcpyAsync(dq, q_host, align_up(qb, 256) + align_up(kb, 256) + kb, cudaMemcpyHostToDevice, st));
   } else {
     HE_CUDA_CHECK(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st));
@@ -969,6 +968,21 @@ int he_decode_step_host_enqueue(const he_config* cfg, const he_cache* cache, con
   if (int rc = he_decode_step(cfg, cache, dq, dk, dv, dvictim, nullptr, nullptr, stream)) return rc;
   HE_CUDA_CHECK(cudaMemcpyAsync(victim_host, dvictim, units * 4, cudaMemcpyDeviceToHost, st));
   return HE_OK;
+}
+
+size_t he_decode_host_block_bytes(const he_config* cfg, size_t offsets[3]) {
+  if (check_config(cfg, true) != HE_OK) return 0;
+  const size_t units = (size_t)cfg->batch * cfg->n_kv_heads;
+  const size_t row = (size_t)cfg->head_dim * esize_of(cfg->dtype);
+  const size_t qb = units * cfg->group_size * row, kb = units * row;
+  if (offsets != nullptr) offsets[0] = 0, offsets[1] = align_up(qb, 256), offsets[2] = align_up(qb, 256) + align_up(kb, 256);
+  return align_up(qb, 256) + align_up(kb, 256) + kb;
+}
+
+int he_decode_step_host_block_enqueue(const he_config* cfg, const he_cache* cache, const void* qkv_host, int32_t* victim_host,
+                                      void* staging, size_t staging_bytes, void* stream) {
+  if (qkv_host == nullptr) return fail(HE_ERR_INVALID_ARG, "qkv_host is null");
+  return he_decode_step_host_enqueue(cfg, cache, qkv_host, nullptr, nullptr, victim_host, staging, staging_bytes, stream);
 }
 
 size_t he_prefill_staging_bytes(const he_config* cfg, int32_t max_prompt_len) {

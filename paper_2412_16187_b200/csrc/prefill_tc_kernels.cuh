@@ -65,7 +65,7 @@ __device__ __forceinline__ uint32_t rt_e4m3_of_int(int v) {
 
 // Byte offsets of the kernel's dynamic shared memory (after rounding its base up to 1024 bytes).
 struct RtLayout {
-  uint32_t a, b, codes, pos, owner, m, m2, rb, dn, qraw, kraw, total;
+  uint32_t a, b, codes, pos, owner, m, m2, rb, ub, ps, dn, qraw, kraw, total;
 };
 // `slots` is the budget rounded up to whole tiles; the tile-maximum table has an odd pitch (conflict-free column writes).
 __host__ __device__ inline int rt_mpitch(int slots, bool table_in_smem) { return table_in_smem ? kRtMaxSlots / kRtTile + 1 : ((slots / kRtTile) | 1); }
@@ -83,6 +83,8 @@ __host__ __device__ inline RtLayout rt_layout(int words, int slots, int G, bool 
   // second-largest key per (step, tile): kept where it fits (tables in shared memory, 8-bit operands)
   L.m2 = o, o += (table_in_smem && fp8) ? (uint32_t)kRtRows * rt_mpitch(slots, true) * 4u : 0u;
   L.rb = o, o += kRtRows * 4u;
+  L.ub = o, o += kRtRows * 4u;
+  L.ps = o, o += kRtRows * 4u;
   L.dn = o, o += kRtRows * kRtRows * 2u;
   L.qraw = o, o += 2u * kRtRows * G * words * 4u;  // two buffers: this block's codes and the next block's
   L.kraw = o, o += 2u * kRtRows * words * 4u;
@@ -183,6 +185,8 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   constexpr int kSecondMaxTiles = 8;  // ... for small tables only: see `second` below
   int32_t* Mx2 = reinterpret_cast<int32_t*>(smem + L.m2);
   int32_t* RB = reinterpret_cast<int32_t*>(smem + L.rb);
+  int32_t* UB = reinterpret_cast<int32_t*>(smem + L.ub);  // per step: no new entry's key can exceed this
+  int32_t* PS = reinterpret_cast<int32_t*>(smem + L.ps);  // per step: the nearest of the 31 steps before it with the same best base slot, or -1
   uint16_t* Dn = reinterpret_cast<uint16_t*>(smem + L.dn);
   uint32_t* qraw = reinterpret_cast<uint32_t*>(smem + L.qraw);
   uint32_t* kraw = reinterpret_cast<uint32_t*>(smem + L.kraw);
@@ -549,11 +553,17 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             Mx[tid * mp + i] = __float2int_rn(mxf);
             if (second) Mx2[tid * mp + i] = __float2int_rn(mxs);
           } else {  // distances of the block's keys: key / 2^14, kept as 16-bit integers
+            // ... and, for step `tid`, the largest distance to any key that enters before it (entries e < tid): whatever
+            // their slots turn out to be, no new entry's key exceeds (that distance, lowest possible slot)
+            float dmax = -1.f;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               uint32_t v[32];
               tc_ld32(taddr + c * 32, v);
               tc_wait_ld();
+#pragma unroll
+              for (int k = 0; k < 32; ++k)
+                if (c * 32 + k < tid) dmax = fmaxf(dmax, __uint_as_float(v[k]));
               uint32_t pk[16];
 #pragma unroll
               for (int k = 0; k < 16; ++k)
@@ -563,6 +573,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
 #pragma unroll
               for (int k = 0; k < 4; ++k) dst[k] = make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
             }
+            UB[tid] = dmax < 0.f ? -1 : ((__float2int_rn(dmax * (1.f / 16384.f)) << kRtKeyShift) | kRtIdxMask);
             if (last_of_handover) {
               tc_fence_before();
               __syncwarp();
@@ -575,6 +586,14 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           int rb = 0;
           for (int i = 0; i < nbase; ++i) rb = max(rb, Mx[tid * mp + i]);
           RB[tid] = rb;
+        }
+        asm volatile("bar.sync 2, 128;" ::: "memory");  // the four reader warps: RB is complete
+        if (ok) {
+          const int mine = RB[tid] & kRtIdxMask;
+          int ps = -1;
+          for (int q = 1; q < 32 && q <= tid; ++q)
+            if (ps < 0 && (RB[tid - q] & kRtIdxMask) == mine) ps = tid - q;
+          PS[tid] = ps;
         }
       }
       it += nsync;
@@ -617,13 +636,65 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
 #pragma unroll
         for (int w = 0; w < WORDS; ++w) kc[w] = kb_codes[w];
         bool scored = !(write_scores && t0 + rows == N);  // only the prompt's last step stores Eq. 5 scores
+        // Without protected windows most steps need no step-to-step chain at all. A step is EASY when its best base key
+        // beats every key a new entry could have (UB) and that base slot still holds its base token: its victim is then
+        // that slot, known from the tile maxima alone. Consecutive easy steps with distinct slots do not influence one
+        // another (each only removes its own slot and adds an entry the later bounds already cover), so a run of up to 32
+        // of them is settled by the warp's lanes side by side. Only the other steps - a stale maximum, a new entry that
+        // may win, the scoring pass - go through the sequential path below, one at a time.
+        constexpr bool FAST = !PROT;
+        bool resume = false;  // re-entering the sequential path at the same step after a repair or the scoring pass
         int r = 0;
         while (r < rows) {
           int status = 0, kn_out = 0;
+          if (FAST && !resume) {
+            for (;;) {
+              const int rr = r + lane;
+              const bool in = rr < rows;
+              const int kbl = in ? RB[rr] : 0;
+              const int sl = kRtIdxMask - (kbl & kRtIdxMask);
+              bool hard = !in || kbl <= UB[in ? rr : 0] || owner[in ? sl : 0] >= 0 || (!scored && rr == rows - 1) || !HE_IN_RANGE(sl, C);
+              hard |= in && PS[rr] >= r;  // an earlier step of the run takes the same slot
+              const unsigned hb = __ballot_sync(0xFFFFFFFFu, hard);
+              const int ne = hb ? __ffs(hb) - 1 : 32;
+              if (ne == 0) break;
+              if (lane < ne) {  // Algorithm 1 lines 2-5 on the table for step rr
+                owner[sl] = (int16_t)rr;
+#pragma unroll
+                for (int w = 0; w < WORDS; ++w) codes_t[sl * WORDS + w] = kb_codes[rr * WORDS + w];
+                pos_t[sl] = t0 + rr;
+              }
+              // the tokens of these steps enter as entries r .. r + ne - 1 (lane e / 4, register e % 4)
+#pragma unroll
+              for (int q4 = 0; q4 < 4; ++q4) {
+                const int src = 4 * lane + q4 - r;
+                const int sv = __shfl_sync(0xFFFFFFFFu, sl, src & 31);
+                if (src >= 0 && src < ne) {
+                  if (q4 == 0) vb0 = kRtIdxMask - sv;
+                  if (q4 == 1) vb1 = kRtIdxMask - sv;
+                  if (q4 == 2) vb2 = kRtIdxMask - sv;
+                  if (q4 == 3) vb3 = kRtIdxMask - sv;
+                }
+              }
+              r += ne;
+              if (GLOBAL_TABLE) __threadfence_block();
+              __syncwarp();
+              if (r >= rows) break;
+            }
+            if (r >= rows) break;
+            // step r takes the sequential path: its operands
+            dd = *reinterpret_cast<const uint2*>(Dn + r * kRtRows + 4 * lane);
+            kb = RB[r];
+            own_kb = owner[kRtIdxMask - (kb & kRtIdxMask)];
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) kc[w] = kb_codes[r * WORDS + w];
+          }
+          resume = false;
+          const int r_end = FAST ? r + 1 : rows;
           // unrolled by two: the carried values (next row's prefetches) change names instead of being copied, which is
           // worth 10-20 % of the loop on this single-warp critical path (measured; unrolling by four is slower again)
 #pragma unroll 2
-          for (; r < rows; ++r) {
+          for (; r < r_end; ++r) {
             const int rn = r + 1 < rows ? r + 1 : r;  // the last step fetches its own row again (unused)
             const uint2 dd_n = *reinterpret_cast<const uint2*>(Dn + rn * kRtRows + 4 * lane);
             const int kb_n = RB[rn];
@@ -679,6 +750,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
 #pragma unroll
             for (int w = 0; w < WORDS; ++w) kc[w] = kc_n[w];
           }
+          if (status != 0) resume = true;
           if (status == 1) {
             // Repair for step r: recompute the maximum of the tile the stale key came from, over the slots that
             // still hold their base token, until the row's best base key is exact (or no longer matters). Each pass

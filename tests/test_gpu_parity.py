@@ -172,6 +172,35 @@ def test_enqueued_host_steps_on_two_streams_match_device_calls():
             assert torch.equal(getattr(ref.gpu, name), getattr(c.gpu, name)), name
 
 
+def test_host_block_steps_match_device_calls():
+    """he_decode_step_host_block_enqueue: a step's q, k, v in one pinned block at the documented offsets, one copy in."""
+    from paper_2412_16187_b200 import decode_staging_bytes
+    w = PARITY_CASES["protected_tiny"]
+    steps = 6
+    ref, x = Case(w), Case(w)
+    for c in (ref, x):
+        c.gpu.prefill_compress(c.dQ, c.dK, c.dV, c.dplen)
+    dq, dk, dv = (wl.gen_decode_inputs(w, n, 0, steps) for n in "qkv")
+    want = [ref.gpu.decode_step(to_dev(dq[i], w), to_dev(dk[i], w), to_dev(dv[i], w)).cpu() for i in range(steps)]
+    nbytes, offs = x.gpu.host_block_layout()
+    assert offs[0] == 0 and offs[1] % 256 == 0 and offs[2] % 256 == 0 and nbytes == offs[2] + dk[0].nbytes
+    block = torch.zeros((steps, (nbytes + 255) // 256 * 256), dtype=torch.uint8).pin_memory()
+    for i in range(steps):
+        for o, t in zip(offs, (dq[i], dk[i], dv[i])):
+            block[i, o:o + t.nbytes] = torch.from_numpy(np.ascontiguousarray(t).view(np.uint8).reshape(-1))
+    st = torch.empty(decode_staging_bytes(x.gpu.cfg), dtype=torch.uint8, device="cuda")
+    got = torch.empty((steps, w.n_seq, w.n_kv_heads), dtype=torch.int32).pin_memory()
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for i in range(steps):
+        x.gpu.decode_step_host_block_enqueue_raw(block[i].data_ptr(), got[i].data_ptr(), st.data_ptr(), st.numel(), stream.cuda_stream)
+    torch.cuda.synchronize()
+    for i in range(steps):
+        assert torch.equal(got[i], want[i]), i
+    for name in ("codes", "pos", "scores", "k_cache", "v_cache", "fill", "next_pos"):
+        assert torch.equal(getattr(ref.gpu, name), getattr(x.gpu, name)), name
+
+
 def _sampled_full_size_check(w, seqs, decode_steps, early_inputs=False):
     """Full-size workload on the device in the launch configuration the benchmark times; the oracle replays only
     the sampled sequences (all their KV heads) on the device's codes and must reproduce their final state."""
