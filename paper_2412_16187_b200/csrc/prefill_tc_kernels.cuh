@@ -30,6 +30,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "hash_tc_kernels.cuh"
 #include "prefill_kernels.cuh"
 
@@ -44,6 +46,7 @@ constexpr int kRtMaxSlotsGlobal = 12288;  // largest budget at all: the tables t
 constexpr int kRtKeyShift = 14;
 constexpr int kRtIdxMask = (1 << kRtKeyShift) - 1;
 constexpr int kRtStaleLimit = 64;  // repairs after which a block is cut short
+constexpr int kRtFastNum = 3, kRtFastDen = 10;  // run-based resolver while fewer than NUM / DEN of a unit's steps are not easy
 constexpr int kRtAtomBytes = kRtRows * 128;  // one 64-column K-major swizzle atom of a 128-row operand tile
 
 __device__ __forceinline__ void tc_mma_f8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
@@ -65,7 +68,7 @@ __device__ __forceinline__ uint32_t rt_e4m3_of_int(int v) {
 
 // Byte offsets of the kernel's dynamic shared memory (after rounding its base up to 1024 bytes).
 struct RtLayout {
-  uint32_t a, b, codes, pos, owner, m, m2, rb, ub, ps, dn, qraw, kraw, total;
+  uint32_t a, b, codes, pos, owner, m, m2, rb, ub, ps, es, dn, qraw, kraw, total;
 };
 // `slots` is the budget rounded up to whole tiles; the tile-maximum table has an odd pitch (conflict-free column writes).
 __host__ __device__ inline int rt_mpitch(int slots, bool table_in_smem) { return table_in_smem ? kRtMaxSlots / kRtTile + 1 : ((slots / kRtTile) | 1); }
@@ -85,6 +88,7 @@ __host__ __device__ inline RtLayout rt_layout(int words, int slots, int G, bool 
   L.rb = o, o += kRtRows * 4u;
   L.ub = o, o += kRtRows * 4u;
   L.ps = o, o += kRtRows * 4u;
+  L.es = o, o += kRtRows * 4u;
   L.dn = o, o += kRtRows * kRtRows * 2u;
   L.qraw = o, o += 2u * kRtRows * G * words * 4u;  // two buffers: this block's codes and the next block's
   L.kraw = o, o += 2u * kRtRows * words * 4u;
@@ -159,7 +163,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   __shared__ __align__(8) unsigned long long bars[4 * NSTAGE];
   __shared__ uint32_t tmem_base_s;
   __shared__ volatile int abort_flag;
-  __shared__ int s_unit, s_done;
+  __shared__ int s_unit, s_done, s_fast;
   __shared__ uint16_t entry_slot[PROT ? kRtRows : 1];  // PROT: the slot each of the block's steps wrote to
   // four code bits -> four bf16 values: operand B takes +-1 (bit set: +1), operand A -+2^13 (bit set: -2^13)
   __shared__ uint2 s_lut_a[16], s_lut_b[16];
@@ -186,7 +190,8 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   int32_t* Mx2 = reinterpret_cast<int32_t*>(smem + L.m2);
   int32_t* RB = reinterpret_cast<int32_t*>(smem + L.rb);
   int32_t* UB = reinterpret_cast<int32_t*>(smem + L.ub);  // per step: no new entry's key can exceed this
-  int32_t* PS = reinterpret_cast<int32_t*>(smem + L.ps);  // per step: the nearest of the 31 steps before it with the same best base slot, or -1
+  int32_t* PS = reinterpret_cast<int32_t*>(smem + L.ps);  // per step: slot of the best base key, flags (see the readers)
+  int32_t* ES = reinterpret_cast<int32_t*>(smem + L.es);  // per new entry of the block: 16383 - its slot while resident
   uint16_t* Dn = reinterpret_cast<uint16_t*>(smem + L.dn);
   uint32_t* qraw = reinterpret_cast<uint32_t*>(smem + L.qraw);
   uint32_t* kraw = reinterpret_cast<uint32_t*>(smem + L.kraw);
@@ -269,6 +274,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     // PROT with the tables in global memory: positions are too far away for the resolver's step-ahead checks, so warp 0
     // keeps the slots of the 32 newest tokens in a register ring (lane l: the newest token congruent to l mod 32; the
     // first C tokens sit in slot = position) and sinks are recognised by their slot (they never leave slots 0..n_sink-1).
+    if (tid == 0) s_fast = PROT ? 0 : 1;  // a unit's first block tries the run-based loop
     int myring = -1;
     if (PROT && GLOBAL_TABLE) {
       const int pl = fill0 - 1 - ((fill0 - 1 - lane) & 31);
@@ -561,9 +567,11 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
               uint32_t v[32];
               tc_ld32(taddr + c * 32, v);
               tc_wait_ld();
+              if (s_fast) {
 #pragma unroll
-              for (int k = 0; k < 32; ++k)
-                if (c * 32 + k < tid) dmax = fmaxf(dmax, __uint_as_float(v[k]));
+                for (int k = 0; k < 32; ++k)
+                  if (c * 32 + k < tid) dmax = fmaxf(dmax, __uint_as_float(v[k]));
+              }
               uint32_t pk[16];
 #pragma unroll
               for (int k = 0; k < 16; ++k)
@@ -587,13 +595,16 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           for (int i = 0; i < nbase; ++i) rb = max(rb, Mx[tid * mp + i]);
           RB[tid] = rb;
         }
-        asm volatile("bar.sync 2, 128;" ::: "memory");  // the four reader warps: RB is complete
-        if (ok) {
+        if (s_fast) asm volatile("bar.sync 2, 128;" ::: "memory");  // the four reader warps: RB and UB are complete
+        if (ok && s_fast) {
+          // what the resolver's easy-run test needs of step `tid`, in one word: the slot of its best base key (14 bits),
+          // whether a new entry might beat that key (bit 14), and how many steps back the nearest earlier step with the
+          // same slot lies (bits 16-20; 0: none among the 31 steps before it)
           const int mine = RB[tid] & kRtIdxMask;
-          int ps = -1;
+          int back = 0;
           for (int q = 1; q < 32 && q <= tid; ++q)
-            if (ps < 0 && (RB[tid - q] & kRtIdxMask) == mine) ps = tid - q;
-          PS[tid] = ps;
+            if (back == 0 && (RB[tid - q] & kRtIdxMask) == mine) back = q;
+          PS[tid] = (kRtIdxMask - mine) | (RB[tid] <= UB[tid] ? (1 << 14) : 0) | (back << 16);
         }
       }
       it += nsync;
@@ -642,223 +653,244 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
         // another (each only removes its own slot and adds an entry the later bounds already cover), so a run of up to 32
         // of them is settled by the warp's lanes side by side. Only the other steps - a stale maximum, a new entry that
         // may win, the scoring pass - go through the sequential path below, one at a time.
-        constexpr bool FAST = !PROT;
-        bool resume = false;  // re-entering the sequential path at the same step after a repair or the scoring pass
-        int r = 0;
-        while (r < rows) {
-          int status = 0, kn_out = 0;
-          if (FAST && !resume) {
-            for (;;) {
-              const int rr = r + lane;
-              const bool in = rr < rows;
-              const int kbl = in ? RB[rr] : 0;
-              const int sl = kRtIdxMask - (kbl & kRtIdxMask);
-              bool hard = !in || kbl <= UB[in ? rr : 0] || owner[in ? sl : 0] >= 0 || (!scored && rr == rows - 1) || !HE_IN_RANGE(sl, C);
-              hard |= in && PS[rr] >= r;  // an earlier step of the run takes the same slot
-              const unsigned hb = __ballot_sync(0xFFFFFFFFu, hard);
-              const int ne = hb ? __ffs(hb) - 1 : 32;
-              if (ne == 0) break;
-              if (lane < ne) {  // Algorithm 1 lines 2-5 on the table for step rr
-                owner[sl] = (int16_t)rr;
-#pragma unroll
-                for (int w = 0; w < WORDS; ++w) codes_t[sl * WORDS + w] = kb_codes[rr * WORDS + w];
-                pos_t[sl] = t0 + rr;
+        // The run test costs about as much as a sequential step and fails at every step that is not easy, so it only
+        // pays while those are few (measured break-even: three steps in ten). Each block counts the steps that were not
+        // easy, whichever loop it ran, and the unit's next block picks its loop by that count; s_fast also tells the
+        // readers whether the next block needs the run test's tables (UB, PS) at all.
+        const bool FAST = !PROT && s_fast != 0;
+        int n_not_easy = 0;
+        // the loop is compiled twice, so that the plain sequential form keeps the tight code it had before the run test
+        auto resolve_block = [&](auto fast_c) {
+          constexpr bool FASTC = decltype(fast_c)::value;
+          bool resume = false;  // re-entering the sequential path at the same step after a repair or the scoring pass
+          bool vb_dirty = false;
+          if (FASTC) {  // no entry of this block is resident yet
+            *reinterpret_cast<int4*>(ES + 4 * lane) = make_int4(kAbsent, kAbsent, kAbsent, kAbsent);
+            __syncwarp();
+          }
+          int r = 0;
+          while (r < rows) {
+            int status = 0, kn_out = 0;
+            if (FASTC && !resume) {
+              if (vb_dirty) {  // the sequential path changed the residency of this lane's entries
+                *reinterpret_cast<int4*>(ES + 4 * lane) = make_int4(vb0, vb1, vb2, vb3);
+                vb_dirty = false;
+                __syncwarp();
               }
-              // the tokens of these steps enter as entries r .. r + ne - 1 (lane e / 4, register e % 4)
-#pragma unroll
-              for (int q4 = 0; q4 < 4; ++q4) {
-                const int src = 4 * lane + q4 - r;
-                const int sv = __shfl_sync(0xFFFFFFFFu, sl, src & 31);
-                if (src >= 0 && src < ne) {
-                  if (q4 == 0) vb0 = kRtIdxMask - sv;
-                  if (q4 == 1) vb1 = kRtIdxMask - sv;
-                  if (q4 == 2) vb2 = kRtIdxMask - sv;
-                  if (q4 == 3) vb3 = kRtIdxMask - sv;
+              for (;;) {
+                const int rr = r + lane;
+                const bool in = rr < rows;
+                const int pk = PS[in ? rr : 0];
+                const int sl = pk & kRtIdxMask, back = pk >> 16;
+                const int own = owner[sl];
+                // not easy: a new entry might win, the slot is no longer its base token's, an earlier step of this run
+                // takes the same slot, or this is the prompt's last step and it still has to store its scores
+                const bool hard = !in | ((pk >> 14) & 1) | (own >= 0) | (back != 0 && back <= lane) | (!scored && rr == rows - 1) |
+                                  !HE_IN_RANGE(sl, C);
+                const unsigned hb = __ballot_sync(0xFFFFFFFFu, hard);
+                const int ne = hb ? __ffs(hb) - 1 : 32;
+                if (ne == 0) break;
+                if (lane < ne) {  // Algorithm 1 lines 2-5 on the table for step rr; its token enters as entry rr
+                  owner[sl] = (int16_t)rr;
+  #pragma unroll
+                  for (int w = 0; w < WORDS; ++w) codes_t[sl * WORDS + w] = kb_codes[rr * WORDS + w];
+                  pos_t[sl] = t0 + rr;
+                  ES[rr] = kRtIdxMask - sl;
+                }
+                r += ne;
+                if (GLOBAL_TABLE) __threadfence_block();
+                __syncwarp();
+                if (r >= rows) break;
+              }
+              if (r >= rows) break;
+              ++n_not_easy;
+              // step r takes the sequential path: its operands, and this lane's entries as the runs left them
+              dd = *reinterpret_cast<const uint2*>(Dn + r * kRtRows + 4 * lane);
+              kb = RB[r];
+              own_kb = owner[kRtIdxMask - (kb & kRtIdxMask)];
+  #pragma unroll
+              for (int w = 0; w < WORDS; ++w) kc[w] = kb_codes[r * WORDS + w];
+              const int4 e4 = *reinterpret_cast<const int4*>(ES + 4 * lane);
+              vb0 = e4.x, vb1 = e4.y, vb2 = e4.z, vb3 = e4.w;
+            }
+            vb_dirty = true;
+            resume = false;
+            const int r_end = FASTC ? r + 1 : rows;
+            // unrolled by two: the carried values (next row's prefetches) change names instead of being copied, which is
+            // worth 10-20 % of the loop on this single-warp critical path (measured; unrolling by four is slower again)
+  #pragma unroll 2
+            for (; r < r_end; ++r) {
+              const int rn = r + 1 < rows ? r + 1 : r;  // the last step fetches its own row again (unused)
+              const uint2 dd_n = *reinterpret_cast<const uint2*>(Dn + rn * kRtRows + 4 * lane);
+              const int kb_n = RB[rn];
+              int own_n = owner[kRtIdxMask - (kb_n & kRtIdxMask)];
+              int act_slot = 0;
+              if (PROT) {  // eligibility of the next step's best base slot at that step; the slot of the entry that turns eligible
+                if (protected_at(kRtIdxMask - (kb_n & kRtIdxMask), t0 + r + 1, 1)) own_n = 0;
+                if (Rn > 0 && r >= Rn) act_slot = entry_slot[r - Rn];
+              }
+              uint32_t kc_n[WORDS];
+  #pragma unroll
+              for (int w = 0; w < WORDS; ++w) kc_n[w] = kb_codes[rn * WORDS + w];
+              // best new entry (inserted by an earlier step of this block and still resident)
+              const int k0 = (int)((dd.x & 0xFFFFu) << kRtKeyShift) + vb0;
+              const int k1 = (int)((dd.x >> 16) << kRtKeyShift) + vb1;
+              const int k2 = (int)((dd.y & 0xFFFFu) << kRtKeyShift) + vb2;
+              const int k3 = (int)((dd.y >> 16) << kRtKeyShift) + vb3;
+              const int kn = __reduce_max_sync(0xFFFFFFFFu, max(max(k0, k1), max(k2, k3)));
+              if (!PROT && !FASTC) n_not_easy += (own_kb >= 0 || kn >= kb) ? 1 : 0;  // (a repaired step re-enters and counts twice)
+              // best base slot: the tile maxima are upper bounds; one that points at an evicted slot needs a repair
+              if (kb > kn && own_kb >= 0) {
+                status = 1;
+                kn_out = kn;
+                break;
+              }
+              if (!scored && r == rows - 1) {
+                status = 2;
+                break;
+              }
+              const int best = max(kb, kn);
+              const int slot = kRtIdxMask - (best & kRtIdxMask);
+              // a new entry that wins leaves: its lane recognises its own key (keys of resident entries are distinct,
+              // absent ones are negative); then this step's token enters as entry r
+              // (with protected windows: the entry of step r - n_recent, which is no longer recent from the next step on)
+              const int e_act = PROT ? r - Rn : r;
+              const bool mine = e_act >= 0 && lane == (e_act >> 2);
+              const int sel = e_act & 3, nv = kRtIdxMask - ((PROT && Rn > 0) ? act_slot : slot);
+              if (PROT) entry_slot[r] = (uint16_t)slot;
+              if (PROT && GLOBAL_TABLE && lane == ((t0 + r) & 31)) myring = slot;
+              vb0 = (mine && sel == 0) ? nv : (k0 == best ? kAbsent : vb0);
+              vb1 = (mine && sel == 1) ? nv : (k1 == best ? kAbsent : vb1);
+              vb2 = (mine && sel == 2) ? nv : (k2 == best ? kAbsent : vb2);
+              vb3 = (mine && sel == 3) ? nv : (k3 == best ? kAbsent : vb3);
+              // Algorithm 1 lines 2-5 on the table (K / V rows follow in the gather kernel). Every lane stores the same
+              // values to the same addresses: no divergent branch, and each lane later reads back its own stores.
+              if (HE_IN_RANGE(slot, C)) {
+                owner[slot] = (int16_t)r;
+  #pragma unroll
+                for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
+                pos_t[slot] = t0 + r;
+              }
+              if (slot == kRtIdxMask - (kb_n & kRtIdxMask)) own_n = r;  // the owner fetched ahead predates this step
+              dd = dd_n, kb = kb_n, own_kb = own_n;
+  #pragma unroll
+              for (int w = 0; w < WORDS; ++w) kc[w] = kc_n[w];
+            }
+            if (status != 0) resume = true;
+            if (status == 1) {
+              // Repair for step r: recompute the maximum of the tile the stale key came from, over the slots that
+              // still hold their base token, until the row's best base key is exact (or no longer matters). Each pass
+              // makes one tile exact, so nbase passes always suffice; the bound only guards against a corrupted table.
+              uint32_t qw[kMaxGroup * WORDS];
+  #pragma unroll
+              for (int i = 0; i < kMaxGroup * WORDS; ++i) qw[i] = i < GW ? qb[r * GW + i] : 0u;
+              const int kn = kn_out;  // the step's best new entry, as the hot loop left it
+              // lane i keeps tile i's maximum for this step in a register (tables in shared memory: at most 32 tiles)
+              int mt = (!GLOBAL_TABLE && lane < nbase) ? Mx[r * mp + lane] : 0;
+              // First the cheap way: the stale key was its tile's largest at the block's start, so the tile's second-largest
+              // key bounds what is left of that tile, and it is exact if its slot still holds its base token. If the
+              // row's best key is then a live slot (or no better than the best new entry) the step is settled without
+              // recomputing a tile.
+              bool settled = false;
+              if (second) {
+                const int cb0 = (kRtIdxMask - (kb & kRtIdxMask)) / kRtTile;
+                mt = lane == cb0 ? Mx2[r * mp + cb0] : mt;
+                kb = __reduce_max_sync(0xFFFFFFFFu, mt);
+                if (kb <= kn) {
+                  settled = true;
+                } else if (kb > 0) {
+                  const int sb = kRtIdxMask - (kb & kRtIdxMask);
+                  bool bad = owner[sb] >= 0;
+                  if (PROT && !bad) {
+                    const int pb = table_pos(sb);
+                    bad = pb < S || pb >= t0 + r - Rn;
+                  }
+                  settled = !bad;
                 }
               }
-              r += ne;
-              if (GLOBAL_TABLE) __threadfence_block();
-              __syncwarp();
-              if (r >= rows) break;
-            }
-            if (r >= rows) break;
-            // step r takes the sequential path: its operands
-            dd = *reinterpret_cast<const uint2*>(Dn + r * kRtRows + 4 * lane);
-            kb = RB[r];
-            own_kb = owner[kRtIdxMask - (kb & kRtIdxMask)];
-#pragma unroll
-            for (int w = 0; w < WORDS; ++w) kc[w] = kb_codes[r * WORDS + w];
-          }
-          resume = false;
-          const int r_end = FAST ? r + 1 : rows;
-          // unrolled by two: the carried values (next row's prefetches) change names instead of being copied, which is
-          // worth 10-20 % of the loop on this single-warp critical path (measured; unrolling by four is slower again)
-#pragma unroll 2
-          for (; r < r_end; ++r) {
-            const int rn = r + 1 < rows ? r + 1 : r;  // the last step fetches its own row again (unused)
-            const uint2 dd_n = *reinterpret_cast<const uint2*>(Dn + rn * kRtRows + 4 * lane);
-            const int kb_n = RB[rn];
-            int own_n = owner[kRtIdxMask - (kb_n & kRtIdxMask)];
-            int act_slot = 0;
-            if (PROT) {  // eligibility of the next step's best base slot at that step; the slot of the entry that turns eligible
-              if (protected_at(kRtIdxMask - (kb_n & kRtIdxMask), t0 + r + 1, 1)) own_n = 0;
-              if (Rn > 0 && r >= Rn) act_slot = entry_slot[r - Rn];
-            }
-            uint32_t kc_n[WORDS];
-#pragma unroll
-            for (int w = 0; w < WORDS; ++w) kc_n[w] = kb_codes[rn * WORDS + w];
-            // best new entry (inserted by an earlier step of this block and still resident)
-            const int k0 = (int)((dd.x & 0xFFFFu) << kRtKeyShift) + vb0;
-            const int k1 = (int)((dd.x >> 16) << kRtKeyShift) + vb1;
-            const int k2 = (int)((dd.y & 0xFFFFu) << kRtKeyShift) + vb2;
-            const int k3 = (int)((dd.y >> 16) << kRtKeyShift) + vb3;
-            const int kn = __reduce_max_sync(0xFFFFFFFFu, max(max(k0, k1), max(k2, k3)));
-            // best base slot: the tile maxima are upper bounds; one that points at an evicted slot needs a repair
-            if (kb > kn && own_kb >= 0) {
-              status = 1;
-              kn_out = kn;
-              break;
-            }
-            if (!scored && r == rows - 1) {
-              status = 2;
-              break;
-            }
-            const int best = max(kb, kn);
-            const int slot = kRtIdxMask - (best & kRtIdxMask);
-            // a new entry that wins leaves: its lane recognises its own key (keys of resident entries are distinct,
-            // absent ones are negative); then this step's token enters as entry r
-            // (with protected windows: the entry of step r - n_recent, which is no longer recent from the next step on)
-            const int e_act = PROT ? r - Rn : r;
-            const bool mine = e_act >= 0 && lane == (e_act >> 2);
-            const int sel = e_act & 3, nv = kRtIdxMask - ((PROT && Rn > 0) ? act_slot : slot);
-            if (PROT) entry_slot[r] = (uint16_t)slot;
-            if (PROT && GLOBAL_TABLE && lane == ((t0 + r) & 31)) myring = slot;
-            vb0 = (mine && sel == 0) ? nv : (k0 == best ? kAbsent : vb0);
-            vb1 = (mine && sel == 1) ? nv : (k1 == best ? kAbsent : vb1);
-            vb2 = (mine && sel == 2) ? nv : (k2 == best ? kAbsent : vb2);
-            vb3 = (mine && sel == 3) ? nv : (k3 == best ? kAbsent : vb3);
-            // Algorithm 1 lines 2-5 on the table (K / V rows follow in the gather kernel). Every lane stores the same
-            // values to the same addresses: no divergent branch, and each lane later reads back its own stores.
-            if (HE_IN_RANGE(slot, C)) {
-              owner[slot] = (int16_t)r;
-#pragma unroll
-              for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
-              pos_t[slot] = t0 + r;
-            }
-            if (slot == kRtIdxMask - (kb_n & kRtIdxMask)) own_n = r;  // the owner fetched ahead predates this step
-            dd = dd_n, kb = kb_n, own_kb = own_n;
-#pragma unroll
-            for (int w = 0; w < WORDS; ++w) kc[w] = kc_n[w];
-          }
-          if (status != 0) resume = true;
-          if (status == 1) {
-            // Repair for step r: recompute the maximum of the tile the stale key came from, over the slots that
-            // still hold their base token, until the row's best base key is exact (or no longer matters). Each pass
-            // makes one tile exact, so nbase passes always suffice; the bound only guards against a corrupted table.
-            uint32_t qw[kMaxGroup * WORDS];
-#pragma unroll
-            for (int i = 0; i < kMaxGroup * WORDS; ++i) qw[i] = i < GW ? qb[r * GW + i] : 0u;
-            const int kn = kn_out;  // the step's best new entry, as the hot loop left it
-            // lane i keeps tile i's maximum for this step in a register (tables in shared memory: at most 32 tiles)
-            int mt = (!GLOBAL_TABLE && lane < nbase) ? Mx[r * mp + lane] : 0;
-            // First the cheap way: the stale key was its tile's largest at the block's start, so the tile's second-largest
-            // key bounds what is left of that tile, and it is exact if its slot still holds its base token. If the
-            // row's best key is then a live slot (or no better than the best new entry) the step is settled without
-            // recomputing a tile.
-            bool settled = false;
-            if (second) {
-              const int cb0 = (kRtIdxMask - (kb & kRtIdxMask)) / kRtTile;
-              mt = lane == cb0 ? Mx2[r * mp + cb0] : mt;
-              kb = __reduce_max_sync(0xFFFFFFFFu, mt);
-              if (kb <= kn) {
-                settled = true;
-              } else if (kb > 0) {
+              for (int pass = 0; !settled && pass <= nbase; ++pass) {
+                ++stale;
+                const int cb = (kRtIdxMask - (kb & kRtIdxMask)) / kRtTile;
+                uint32_t hw[kRtTile / 32][WORDS];
+                int ow[kRtTile / 32];  // < 0: the slot still holds its base token (and, PROT, that token is eligible now)
+  #pragma unroll
+                for (int i = 0; i < kRtTile / 32; ++i) {
+                  const int j = cb * kRtTile + lane + 32 * i;  // below smem_slots: rows past the budget hold zeros
+                  ow[i] = j < C ? (int)owner[j] : 0;
+                  if (PROT && j < C) {
+                    const int pj = table_pos(j);
+                    if (pj < S || pj >= t0 + r - Rn) ow[i] = 0;
+                  }
+  #pragma unroll
+                  for (int w = 0; w < WORDS; ++w) hw[i][w] = j < C ? table_word(j * WORDS + w) : 0u;
+                }
+                int km = 0;
+  #pragma unroll
+                for (int i = 0; i < kRtTile / 32; ++i) {
+                  int D = 0;
+  #pragma unroll
+                  for (int g = 0; g < kMaxGroup; ++g) {
+                    if (g < G) {
+  #pragma unroll
+                      for (int w = 0; w < WORDS; ++w) D += __popc(hw[i][w] ^ qw[g * WORDS + w]);
+                    }
+                  }
+                  const int key = (D << kRtKeyShift) + (kRtIdxMask - (cb * kRtTile + lane + 32 * i));
+                  km = max(km, ow[i] < 0 ? key : 0);
+                }
+                km = __reduce_max_sync(0xFFFFFFFFu, km);
+                int rowmax;
+                if (GLOBAL_TABLE) {
+                  Mx[r * mp + cb] = km;  // same value from every lane
+                  rowmax = 0;
+                  for (int i = lane; i < nbase; i += 32) rowmax = max(rowmax, Mx[r * mp + i]);
+                } else {
+                  mt = lane == cb ? km : mt;
+                  rowmax = mt;
+                }
+                kb = __reduce_max_sync(0xFFFFFFFFu, rowmax);
+                if (kb <= kn) break;
                 const int sb = kRtIdxMask - (kb & kRtIdxMask);
                 bool bad = owner[sb] >= 0;
                 if (PROT && !bad) {
                   const int pb = table_pos(sb);
                   bad = pb < S || pb >= t0 + r - Rn;
                 }
-                settled = !bad;
+                if (!bad) break;
               }
-            }
-            for (int pass = 0; !settled && pass <= nbase; ++pass) {
-              ++stale;
-              const int cb = (kRtIdxMask - (kb & kRtIdxMask)) / kRtTile;
-              uint32_t hw[kRtTile / 32][WORDS];
-              int ow[kRtTile / 32];  // < 0: the slot still holds its base token (and, PROT, that token is eligible now)
-#pragma unroll
-              for (int i = 0; i < kRtTile / 32; ++i) {
-                const int j = cb * kRtTile + lane + 32 * i;  // below smem_slots: rows past the budget hold zeros
-                ow[i] = j < C ? (int)owner[j] : 0;
-                if (PROT && j < C) {
-                  const int pj = table_pos(j);
-                  if (pj < S || pj >= t0 + r - Rn) ow[i] = 0;
+              own_kb = -1;  // exact for this step (or below the best new entry)
+              if (stale >= kRtStaleLimit && r + 1 < rows && scored) {  // many repairs: this block ends with step r
+                // finish step r here, then stop
+                const int best = max(kb, kn);
+                const int slot = kRtIdxMask - (best & kRtIdxMask);
+                if (HE_IN_RANGE(slot, C)) {
+                  owner[slot] = (int16_t)r;
+  #pragma unroll
+                  for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
+                  pos_t[slot] = t0 + r;
                 }
-#pragma unroll
-                for (int w = 0; w < WORDS; ++w) hw[i][w] = j < C ? table_word(j * WORDS + w) : 0u;
+                if (PROT && GLOBAL_TABLE && lane == ((t0 + r) & 31)) myring = slot;
+                done = r + 1;
+                break;
               }
-              int km = 0;
-#pragma unroll
-              for (int i = 0; i < kRtTile / 32; ++i) {
-                int D = 0;
-#pragma unroll
-                for (int g = 0; g < kMaxGroup; ++g) {
-                  if (g < G) {
-#pragma unroll
-                    for (int w = 0; w < WORDS; ++w) D += __popc(hw[i][w] ^ qw[g * WORDS + w]);
-                  }
-                }
-                const int key = (D << kRtKeyShift) + (kRtIdxMask - (cb * kRtTile + lane + 32 * i));
-                km = max(km, ow[i] < 0 ? key : 0);
+            } else if (status == 2) {  // Eq. 5 for every slot as the prompt's last step sees the table
+              const uint32_t* qr = qb + r * GW;
+              for (int j = lane; j < C; j += 32) {
+                uint32_t hj[WORDS];
+  #pragma unroll
+                for (int w = 0; w < WORDS; ++w) hj[w] = table_word(j * WORDS + w);
+                sc[j] = -(float)rt_dist<WORDS>(hj, qr, G);
               }
-              km = __reduce_max_sync(0xFFFFFFFFu, km);
-              int rowmax;
-              if (GLOBAL_TABLE) {
-                Mx[r * mp + cb] = km;  // same value from every lane
-                rowmax = 0;
-                for (int i = lane; i < nbase; i += 32) rowmax = max(rowmax, Mx[r * mp + i]);
-              } else {
-                mt = lane == cb ? km : mt;
-                rowmax = mt;
-              }
-              kb = __reduce_max_sync(0xFFFFFFFFu, rowmax);
-              if (kb <= kn) break;
-              const int sb = kRtIdxMask - (kb & kRtIdxMask);
-              bool bad = owner[sb] >= 0;
-              if (PROT && !bad) {
-                const int pb = table_pos(sb);
-                bad = pb < S || pb >= t0 + r - Rn;
-              }
-              if (!bad) break;
+              scored = true;
             }
-            own_kb = -1;  // exact for this step (or below the best new entry)
-            if (stale >= kRtStaleLimit && r + 1 < rows && scored) {  // many repairs: this block ends with step r
-              // finish step r here, then stop
-              const int best = max(kb, kn);
-              const int slot = kRtIdxMask - (best & kRtIdxMask);
-              if (HE_IN_RANGE(slot, C)) {
-                owner[slot] = (int16_t)r;
-#pragma unroll
-                for (int w = 0; w < WORDS; ++w) codes_t[slot * WORDS + w] = kc[w];
-                pos_t[slot] = t0 + r;
-              }
-              if (PROT && GLOBAL_TABLE && lane == ((t0 + r) & 31)) myring = slot;
-              done = r + 1;
-              break;
-            }
-          } else if (status == 2) {  // Eq. 5 for every slot as the prompt's last step sees the table
-            const uint32_t* qr = qb + r * GW;
-            for (int j = lane; j < C; j += 32) {
-              uint32_t hj[WORDS];
-#pragma unroll
-              for (int w = 0; w < WORDS; ++w) hj[w] = table_word(j * WORDS + w);
-              sc[j] = -(float)rt_dist<WORDS>(hj, qr, G);
-            }
-            scored = true;
           }
+        };
+        if (FAST) resolve_block(std::true_type{}); else resolve_block(std::false_type{});
+        if (lane == 0) {
+          s_done = done;
+          // (the sequential loop sees only part of what makes a step not easy, hence its stricter bar for switching back)
+          s_fast = !PROT && (FAST ? n_not_easy * kRtFastDen < done * kRtFastNum : n_not_easy * 10 < done);
         }
-        if (lane == 0) s_done = done;
       } else if (tn < N) {
         const int nrows = (N - tn) < kRtRows ? (N - tn) : kRtRows;
         stage_codes(cur ^ 1, tn, nrows, tid - 32, NT - 32);
