@@ -62,6 +62,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// Bounded wait that neither reads nor raises the abort flag: used on the way out of an aborted CTA, to let work that
+// is already in flight finish before shared or tensor memory is given up. Gives up silently after the same limit.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kTcSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return;
+}
+
 // Bounded wait on two barriers at once: both are polled in the same loop, so their latencies overlap (one polling
 // round trip costs a couple of hundred cycles even when the phase has long completed).
 __device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b,
@@ -249,7 +256,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   constexpr int kAccCols = 3 * N;                          // one accumulator: the three terms side by side
   constexpr int kTmemCols = 2 * kAccCols <= 256 ? 256 : 512;  // two accumulators, rounded up to a power of two
   extern __shared__ unsigned char tc_smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[2 * kTcStages + 4];
+  __shared__ __align__(8) unsigned long long bars[2 * kTcStages + 5];  // the last one: drain barrier of the abort path
   __shared__ uint32_t tmem_base_s;
   __shared__ volatile int abort_flag;
   __shared__ int s_len[kTcLenCache], s_bud[kTcLenCache];
@@ -275,9 +282,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   auto empty_bar = [&](int s) { return bar0 + 8u * (kTcStages + s); };
   auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kTcStages + a); };
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kTcStages + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * kTcStages + 4);
 
   if (tid == 0) {
     abort_flag = 0;
+    mbar_init(drain_bar, 1);
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(full_bar(s), TMA ? 1 : 32);  // TMA: one arrive + byte count; cp.async: every producer lane arrives
       mbar_init(empty_bar(s), 1);  // tcgen05.commit
@@ -363,6 +372,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
           tma_load_4d(smem_u32(As + s * a_stage_bytes + kh * a_half_bytes), &tmap, kh * 64, (int)tl.row0, tl.c2, tl.c3, full_bar(s));
         ++it;
       }
+      // A CTA that gives up must not hand its shared memory back while a tile copy into it is still under way: wait
+      // (bounded) for the copies of the stages armed last.
+      if (abort_flag)
+        for (int u = it > kTcStages ? it - kTcStages : 0; u < it; ++u) mbar_drain(full_bar(u % kTcStages), (u / kTcStages) & 1);
     }
   } else if (warp == 4) {
     // ------------------------------------------------------------------ producer (cp.async fallback)
@@ -432,6 +445,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
         tc_commit(empty_bar(s));    // the stage may be refilled once these MMAs have read it
         tc_commit(tfull_bar(acc));  // and the accumulator is complete
         ++it;
+      }
+      // ... nor free tensor memory under an MMA that is still writing it: one more commit tracks everything this thread
+      // has issued, and its completion is awaited (bounded) before the CTA goes on to the deallocation.
+      if (abort_flag) {
+        tc_commit(drain_bar);
+        mbar_drain(drain_bar, 0);
       }
     }
   } else {

@@ -160,7 +160,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   constexpr int NSYNC = NSTAGE / TP;         // hand-over slots: stage pair (or stage) + accumulator pair (or accumulator)
   constexpr int NT = kRtThreads;
   extern __shared__ unsigned char rt_smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[4 * NSTAGE];
+  __shared__ __align__(8) unsigned long long bars[4 * NSTAGE + 1];  // the last one: drain barrier of the abort path
   __shared__ uint32_t tmem_base_s;
   __shared__ volatile int abort_flag;
   __shared__ int s_unit, s_done, s_fast;
@@ -203,6 +203,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   auto tempty_bar = [&](int x) { return bar0 + 8u * (3 * NSTAGE + x); };  // readers -> MMA: accumulator x is drained
   if (tid == 0) {
     abort_flag = 0;
+    mbar_init(bar0 + 8u * (4 * NSTAGE), 1);
     for (int s = 0; s < NSTAGE; ++s) {
       mbar_init(full_bar(s), 4 * TP);  // one arrival per expander warp
       mbar_init(tfull_bar(s), 1);
@@ -924,6 +925,14 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     __syncthreads();  // the tables and s_unit are reused by the next unit
   }
 
+  // A CTA that gave up must not free tensor memory under an MMA that is still writing it (the operands are written by
+  // this CTA's own threads, so no copy from outside is ever in flight): one more commit tracks everything the MMA thread
+  // has issued, and its completion is awaited (bounded) first.
+  if (abort_flag && warp == kRtMmaWarp && lane == 0) {
+    const uint32_t drain_bar = bar0 + 8u * (4 * NSTAGE);
+    tc_commit(drain_bar);
+    mbar_drain(drain_bar, 0);
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == kRtMmaWarp) {
