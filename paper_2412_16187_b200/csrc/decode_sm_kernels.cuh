@@ -35,8 +35,10 @@ constexpr int kSmUnits = 4;         // units per CTA at most
 constexpr int kSmStages = 8;        // 16-byte code vectors in flight per thread
 constexpr int kSmRowBatch = 5;      // CUDA-core projection: rows per thread and pass (G = 4 queries + the key)
 constexpr int kSmPassRows = 20;     // CUDA-core projection: rows staged per pass (four units of five rows)
-constexpr int kSmMmaRows = 48;      // tensor-core projection: staged rows (4 units x 9 rows at most, in tiles of 16)
-constexpr int kSmMmaStride = 320;   // ... bytes between staged rows: 256 of data, padded so fragment reads spread over the banks
+constexpr int kSmMmaRows = 40;      // tensor-core projection: staged rows (4 units x 9 rows at most, in tiles of 8)
+constexpr int kSmMmaStride = 288;   // ... bytes between staged rows: 256 of data + 32, so that 8-byte fragment reads of a
+                                    // half-warp (4 rows x 4 lanes) fall into 32 different banks
+constexpr int kSmPartStride = 68;   // ... words between rows of the partial-sum table (conflict-free fragment stores)
 constexpr int kSmSchedShift = 21;   // DecodeArgs::sched word = sequence << 21 | budget
 
 struct SmLayout {
@@ -49,7 +51,8 @@ __host__ __device__ inline SmLayout sm_layout(int d, int words, int es, bool mma
   const int nch = (d + kChunk - 1) / kChunk;
   const size_t ring_bytes = (size_t)kSmStages * kSmThreads * 16;
   const size_t xs_bytes = mma ? (size_t)kSmMmaRows * kSmMmaStride : (size_t)kSmPassRows * d * sizeof(float);
-  const size_t part_bytes = mma ? 0 : (size_t)kSmPassRows * nch * 32 * words * sizeof(float);
+  const size_t part_bytes = mma ? (size_t)4 * kSmMmaRows * kSmPartStride * sizeof(float)
+                                : (size_t)kSmPassRows * nch * 32 * words * sizeof(float);
   L.ring = 0;
   L.xs = 0;
   L.part = xs_bytes;
@@ -199,20 +202,29 @@ __global__ void __launch_bounds__(kSmThreads, 2) decode_step_sm_kernel(const Dec
   const int nitems = nch * BP;
   const int groups = NT / nitems;
   const int item = tid % nitems, grp = tid / nitems;
-  // tensor cores: a warp owns 8 bits (n-tile warp % 8) of every 16-row tile warp / 8, warp / 8 + 2, ...; lane = (g, tg)
-  // holds W[channel(ks, tg, j)][8 * nt + g] for its four channels j of each 16-channel step ks
-  const int n_tiles = (b + 7) >> 3, nt = warp & 7, g = lane >> 2, tg = lane & 3;
-  float wreg[kChunk];
+  // tensor cores: D[bit][row] = sum_ch W[ch][bit] x[row][ch] with the BITS as the instruction's M (tiles of 16) and the
+  // step's rows as its N (tiles of 8): 20 rows are three N-tiles instead of two half-empty M-tiles, and a warp's
+  // fragments of W serve all of them. Warp (mt, kq) = (warp % 4, warp / 4) owns bits 16 mt .. 16 mt + 15 and the
+  // 16-channel steps kq and kq + 4; lane (g, tg) holds W[16 ks + 4 tg + j][16 mt + g (+ 8)], j < 4: inside a step a
+  // lane's four channels stand in for the instruction's k = 2 tg, 2 tg + 1, 2 tg + 8, 2 tg + 9 (the order of the terms
+  // of a dot product is free, and the rows are read with the same assignment).
+  const int m_tiles = (b + 15) >> 4, mt = warp & 3, kq = warp >> 2, g = lane >> 2, tg = lane & 3;
+  const int nks = d >> 4;
+  float wreg[MMA ? 16 : kChunk];
   {
     if (MMA) {
-      const int bit = 8 * nt + g;
-      const bool on = nt < n_tiles && bit < b;  // columns beyond b count as zeros
-      const float* wb = W_in + (size_t)(8 * tg) * b + bit;
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
+      for (int h2 = 0; h2 < 2; ++h2) {  // this warp's first and second step
+        const int ks = kq + 4 * h2;
 #pragma unroll
-        for (int j = 0; j < 4; ++j)  // channel 32 (ks / 2) + 8 tg + 4 (ks % 2) + j; d is a multiple of 32
-          wreg[ks * 4 + j] = (on && (ks >> 1) * 32 < d) ? __ldg(wb + ((ks >> 1) * 32 + 4 * (ks & 1) + j) * b) : 0.f;
+        for (int hb = 0; hb < 2; ++hb) {  // bit g, bit g + 8
+          const int bit = 16 * mt + g + 8 * hb;
+          const bool on = mt < m_tiles && ks < nks && bit < b;  // columns beyond b count as zeros
+          const float* wb = W_in + (size_t)(16 * ks + 4 * tg) * b + bit;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) wreg[(h2 * 2 + hb) * 4 + j] = on ? __ldg(wb + j * b) : 0.f;
+        }
+      }
     } else if (grp < groups) {
       const int c0 = (item / BP) * kChunk, bi = item % BP;
       const float* wp = W_in + (size_t)c0 * b + bi;
@@ -221,7 +233,7 @@ __global__ void __launch_bounds__(kSmThreads, 2) decode_step_sm_kernel(const Dec
       for (int cc = 0; cc < kChunk; ++cc) wreg[cc] = on ? __ldg(wp + cc * b) : 0.f;
     }
   }
-  // The new K and V rows wait in shared memory until the victims are known.
+
   // A warp copies a row, a lane 16 bytes of it (no per-thread index arithmetic).
   if (warp < 2 * n_mine) {
     const int i = warp >> 1;
@@ -236,6 +248,9 @@ __global__ void __launch_bounds__(kSmThreads, 2) decode_step_sm_kernel(const Dec
                                 : static_cast<const char*>(k_in) + (size_t)unit * d * es;
       for (int ch = lane; ch < cpr; ch += 32) cp_async16(xs_raw + p * kSmMmaStride + ch * 16, reinterpret_cast<const uint4*>(src) + ch);
     }
+    // rows that only pad the last tile of 8: zeros (their sums are never read)
+    for (int p = rows_total + warp; p < ((rows_total + 7) & ~7); p += NW)
+      for (int ch = lane; ch < cpr; ch += 32) *reinterpret_cast<uint4*>(xs_raw + p * kSmMmaStride + ch * 16) = make_uint4(0u, 0u, 0u, 0u);
   }
   cp_async_commit();
 
@@ -261,62 +276,89 @@ __global__ void __launch_bounds__(kSmThreads, 2) decode_step_sm_kernel(const Dec
     }
     cp_async_commit();
   };
+  // The first round of the ring is addressed before the wait, so that only the copies themselves follow it.
+  const uint4* first[kSmStages];
+  auto plan_ring = [&]() {
+#pragma unroll
+    for (int sl = 0; sl < kSmStages; ++sl) {
+      while (irem == 0 && iu + 1 < n_mine) {
+        ++iu;
+        const int nv = su[iu].nvec;
+        irem = nv > tid ? (nv - tid + NT - 1) / NT : 0;
+        iptr = su[iu].cvec + tid;
+      }
+      first[sl] = irem > 0 ? iptr : nullptr;
+      if (irem > 0) iptr += NT, --irem;
+    }
+  };
   auto fill_ring = [&]() {
 #pragma unroll
-    for (int sl = 0; sl < kSmStages; ++sl) issue_at(rbase + sl * NT * 16);
+    for (int sl = 0; sl < kSmStages; ++sl) {
+      if (first[sl] != nullptr)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(rbase + sl * NT * 16), "l"(first[sl]) : "memory");
+      cp_async_commit();
+    }
   };
   cp_async_wait_all();  // the staged rows have landed
 
   // ---- Eq. 2 on the units' G query rows and key row
   if (MMA) {
     __syncthreads();
-    if (nt < n_tiles) {
-      for (int mt = warp >> 3; mt * 16 < rows_total; mt += NW / 8) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        const int p0 = mt * 16 + g, p1 = p0 + 8;
-        const unsigned char* x0 = xs_raw + p0 * kSmMmaStride + tg * 16;
-        const unsigned char* x1 = xs_raw + p1 * kSmMmaStride + tg * 16;
-        const bool v0 = p0 < rows_total, v1 = p1 < rows_total;  // absent rows count as zeros
+    const int n_tiles = (rows_total + 7) >> 3;  // at most 5
+    if (mt < m_tiles && kq < nks) {
+      float acc[5][4];
 #pragma unroll
-        for (int kp = 0; kp < 4; ++kp) {
-          if (kp * 32 >= d) break;
-          // 16 bytes = channels 32 kp + 8 tg + 0..7: the first half feeds step 2 kp, the second step 2 kp + 1. Inside a
-          // step a lane's four channels stand in for the instruction's k = 2 tg, 2 tg + 1, 2 tg + 8, 2 tg + 9; W follows
-          // the same assignment, and the order of the terms of a dot product is free.
-          const uint4 r0 = v0 ? *reinterpret_cast<const uint4*>(x0 + kp * 64) : make_uint4(0u, 0u, 0u, 0u);
-          const uint4 r1 = v1 ? *reinterpret_cast<const uint4*>(x1 + kp * 64) : make_uint4(0u, 0u, 0u, 0u);
+      for (int n = 0; n < 5; ++n)
 #pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            const int ks = 2 * kp + hf;
-            float w0 = wreg[ks * 4], w1 = wreg[ks * 4 + 1], w2 = wreg[ks * 4 + 2], w3 = wreg[ks * 4 + 3];
-            uint32_t bt[3][2];
+        for (int j = 0; j < 4; ++j) acc[n][j] = 0.f;
 #pragma unroll
-            for (int term = 0; term < 3; ++term) {
-              bt[term][0] = split_bf16x2(w0, w1);
-              bt[term][1] = split_bf16x2(w2, w3);
-            }
-            const uint32_t a0 = hf ? r0.z : r0.x, a2 = hf ? r0.w : r0.y, a1 = hf ? r1.z : r1.x, a3 = hf ? r1.w : r1.y;
+      for (int h2 = 0; h2 < 2; ++h2) {
+        const int ks = kq + 4 * h2;
+        if (ks >= nks) break;
+        // three exact bf16 terms of this step's fragment of W: a0 = (bit g; k 2tg, 2tg+1), a1 = (bit g + 8; same k),
+        // a2 = (bit g; k 2tg + 8, + 9), a3 = (bit g + 8; same)
+        float w00 = wreg[h2 * 8 + 0], w01 = wreg[h2 * 8 + 1], w02 = wreg[h2 * 8 + 2], w03 = wreg[h2 * 8 + 3];
+        float w10 = wreg[h2 * 8 + 4], w11 = wreg[h2 * 8 + 5], w12 = wreg[h2 * 8 + 6], w13 = wreg[h2 * 8 + 7];
+        uint32_t at[3][4];
 #pragma unroll
-            for (int term = 2; term >= 0; --term) mma_bf16_16816(acc, a0, a1, a2, a3, bt[term][0], bt[term][1]);
-          }
+        for (int term = 0; term < 3; ++term) {
+          at[term][0] = split_bf16x2(w00, w01);
+          at[term][1] = split_bf16x2(w10, w11);
+          at[term][2] = split_bf16x2(w02, w03);
+          at[term][3] = split_bf16x2(w12, w13);
         }
-        // sign bits: lane (g, tg) holds rows g and g + 8, bits 2 tg and 2 tg + 1 of the tile; one byte per (row, tile)
-        uint32_t bal[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) bal[j] = __ballot_sync(0xFFFFFFFFu, acc[j] >= 0.f);
-        if (lane < 16) {
-          const int rr = lane & 7, hi = lane >> 3;
-          const uint32_t ev = ((hi ? bal[2] : bal[0]) >> (4 * rr)) & 0xFu, od = ((hi ? bal[3] : bal[1]) >> (4 * rr)) & 0xFu;
-          auto spread = [](uint32_t x) { return (x & 1u) | ((x & 2u) << 1) | ((x & 4u) << 2) | ((x & 8u) << 3); };
-          uint32_t byte = spread(ev) | (spread(od) << 1);
-          const int left = b - 8 * nt;
-          if (left < 8) byte &= (1u << left) - 1u;
-          const int p = mt * 16 + hi * 8 + rr;
-          if (p < rows_total) {
-            const int i = p / R, row = p - i * R;
-            reinterpret_cast<unsigned char*>(&codes_s[i][row * WORDS])[nt] = (unsigned char)byte;
-          }
+        for (int n = 0; n < 5; ++n) {
+          if (n >= n_tiles) break;
+          // row 8 n + g, channels 16 ks + 4 tg + 0..3: 8 bytes
+          const uint2 xv = *reinterpret_cast<const uint2*>(xs_raw + (8 * n + g) * kSmMmaStride + (16 * ks + 4 * tg) * 2);
+#pragma unroll
+          for (int term = 2; term >= 0; --term)  // smallest term first
+            mma_bf16_16816(acc[n], at[term][0], at[term][1], at[term][2], at[term][3], xv.x, xv.y);
         }
+      }
+      // partial sums of this warp's channel steps: P[kq][row][bit]
+#pragma unroll
+      for (int n = 0; n < 5; ++n) {
+        if (n >= n_tiles) break;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          part[((kq * kSmMmaRows) + 8 * n + 2 * tg + (j & 1)) * kSmPartStride + 16 * mt + g + 8 * (j >> 1)] = acc[n][j];
+      }
+    }
+    __syncthreads();
+    // sign bits: a warp takes a row, a lane the bits lane and lane + 32; the steps' partial sums are added in order
+    const int nkq = nks < 4 ? nks : 4;
+    for (int p = warp; p < rows_total; p += NW) {
+      const int i = p / R, row = p - i * R;
+#pragma unroll
+      for (int w = 0; w < WORDS; ++w) {
+        const int bit = 32 * w + lane;
+        float tot = 0.f;
+        if (bit < 16 * m_tiles)
+          for (int q4 = 0; q4 < nkq; ++q4) tot += part[(q4 * kSmMmaRows + p) * kSmPartStride + bit];
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, tot >= 0.f) & word_mask(b, w);
+        if (lane == 0) codes_s[i][row * WORDS + w] = word;
       }
     }
     __syncthreads();
@@ -376,6 +418,7 @@ __global__ void __launch_bounds__(kSmThreads, 2) decode_step_sm_kernel(const Dec
   __syncthreads();
 
   // ---- everything below may depend on the previous kernel of the stream
+  plan_ring();
   cta_griddep_wait(warp);
   fill_ring();
   // counters: every thread reads the fill of its CTA's units itself (no barrier between the wait and the scan); the
@@ -387,10 +430,11 @@ __global__ void __launch_bounds__(kSmThreads, 2) decode_step_sm_kernel(const Dec
     fl[i] = i < n_mine ? __ldcg(su[i].fill_p) : 0;
     tt[i] = (i < n_mine && (prot || i == warp)) ? __ldcg(su[i].npos_p) : 0;
   }
-  for (int idx = tid; idx < n_mine * G * WORDS; idx += NT) {
-    const int i = idx / (G * WORDS), w = idx - i * G * WORDS;
-    if (su[i].qcodes_p != nullptr) su[i].qcodes_p[w] = codes_s[i][w];
-  }
+  if (su[0].qcodes_p != nullptr)  // (all units or none)
+    for (int idx = tid; idx < n_mine * G * WORDS; idx += NT) {
+      const int i = idx / (G * WORDS), w = idx - i * G * WORDS;
+      su[i].qcodes_p[w] = codes_s[i][w];
+    }
 
   // ---- Eq. 5 / Eq. 6: every thread walks its vectors of each unit in turn; the ring delivers them in that order
   const bool write_scores = (flags & HE_FLAG_WRITE_SCORES) != 0;
