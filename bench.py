@@ -141,7 +141,7 @@ def oracle_sample(w, seqs, decode_steps, threads):
     """Times the CPU oracle, as it stands, on the first `seqs` sequences: prefill then `decode_steps` steps."""
     import oracle
 
-    ws = w.scaled(batch=seqs, layers=1)
+    seqs = min(seqs, w.n_seq)
     budgets, plens = w.budgets()[:seqs], w.prompt_lens()[:seqs]
     Nmax = int(plens.max())
     W = wl.gen_W(w)
