@@ -17,6 +17,8 @@ struct HashJob {
   int mode;  // 0: flat rows; 1: prompt keys; 2: prompt queries
   int dtype, d, b;
   long long rows, row_stride;  // mode 0
+  const void* x2;              // mode 0, tensor-core kernel only: a second range of rows2 rows with the same stride, hashed by
+  long long rows2;             //   the same launch; its codes follow the first range's in `out`
   long long s0, s1, s2;        // modes 1, 2: element strides (batch, head, token)
   int heads, G, Hkv;           // heads = heads per sequence of this tensor
   long long Nmax;

@@ -173,6 +173,7 @@ struct TcTile {
   int nrows;
   long long out_base, out_stride;
   int c2, c3;  // tensor-map coordinates of the segment (head, sequence)
+  int second;  // flat rows: the tile lies in the job's second range (its own tensor map)
 };
 
 // Dense schedule (prompt modes, batch within kTcLenCache): s_pref[s] counts the non-empty tiles of the sequences before
@@ -210,12 +211,16 @@ __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long lo
     ti = t % tiles_per_seg;
   }
   long long r_begin, r_end;
+  o->second = 0;
   if (job.mode == 0) {
-    o->base = static_cast<const char*>(job.x);
+    const long long tiles1 = (job.rows + kTcRows - 1) / kTcRows;
+    o->second = ti >= tiles1 ? 1 : 0;
+    if (o->second) ti -= tiles1;
+    o->base = static_cast<const char*>(o->second ? job.x2 : job.x);
     o->stride = job.row_stride;
     r_begin = 0;
-    r_end = job.rows;
-    o->out_base = 0;
+    r_end = o->second ? job.rows2 : job.rows;
+    o->out_base = o->second ? job.rows * WORDS : 0;
     o->out_stride = WORDS;
     o->c2 = 0;
     o->c3 = 0;
@@ -251,7 +256,8 @@ __device__ __forceinline__ bool tc_tile(const HashJob& job, long long t, long lo
 template <int WORDS, bool TMA>
 __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJob job, long long total_tiles,
                                                                      long long tiles_per_seg,
-                                                                     const __grid_constant__ CUtensorMap tmap) {
+                                                                     const __grid_constant__ CUtensorMap tmap,
+                                                                     const __grid_constant__ CUtensorMap tmap2) {
   constexpr int N = 32 * WORDS;
   constexpr int kAccCols = 3 * N;                          // one accumulator: the three terms side by side
   constexpr int kTmemCols = 2 * kAccCols <= 256 ? 256 : 512;  // two accumulators, rounded up to a power of two
@@ -369,7 +375,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
         mbar_arrive_expect_tx(full_bar(s), (uint32_t)a_stage_bytes);
         // rows past the tensor's extent are filled with zeros by the copy engine; their codes are not stored
         for (int kh = 0; kh < KH; ++kh)
-          tma_load_4d(smem_u32(As + s * a_stage_bytes + kh * a_half_bytes), &tmap, kh * 64, (int)tl.row0, tl.c2, tl.c3, full_bar(s));
+          tma_load_4d(smem_u32(As + s * a_stage_bytes + kh * a_half_bytes), tl.second ? &tmap2 : &tmap, kh * 64, (int)tl.row0, tl.c2,
+                      tl.c3, full_bar(s));
         ++it;
       }
       // A CTA that gives up must not hand its shared memory back while a tile copy into it is still under way: wait

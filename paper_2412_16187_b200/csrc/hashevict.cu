@@ -232,16 +232,34 @@ int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments
   if (max_rows_per_segment <= 0 || segments <= 0) return HE_OK;
   const int Wd = words_of(job.b);
   const long long tiles = (max_rows_per_segment + kHashRows - 1) / kHashRows;
-  if (tc_enabled() && job.dtype == HE_DTYPE_BF16 && (job.d == 64 || job.d == 128) && tiles * segments >= 64) {
+  // flat rows may come as two ranges (the decode step's query rows and key rows): one launch of the tensor-core kernel
+  const bool two = job.mode == 0 && job.x2 != nullptr && job.rows2 > 0;
+  const long long tiles2 = two ? (job.rows2 + kHashRows - 1) / kHashRows : 0;
+  const bool tc = tc_enabled() && job.dtype == HE_DTYPE_BF16 && (job.d == 64 || job.d == 128) && (tiles + tiles2) * segments >= 64;
+  if (two && !tc) {  // the CUDA-core kernel takes one range at a time
+    HashJob j1 = job, j2 = job;
+    j1.x2 = nullptr, j1.rows2 = 0;
+    j2.x = job.x2, j2.rows = job.rows2, j2.out = job.out + job.rows * Wd, j2.x2 = nullptr, j2.rows2 = 0;
+    if (int rc = launch_hash(j1, j1.rows, 1, stream, image_built, pdl)) return rc;
+    return launch_hash(j2, j2.rows, 1, stream, image_built, true);
+  }
+  if (tc) {
     static_assert(kTcRows == kHashRows, "both kernels tile rows by 128");
     const int N = 32 * Wd, KH = job.d / 64;
     const size_t smem = 1024 + (size_t)3 * KH * N * 128 + (size_t)kTcStages * KH * kTcRows * 128;
     int sms = 0;
     if (int rc = sm_count(&sms)) return rc;
-    const long long total = tiles * segments;
+    const long long total = tiles * segments + tiles2;
     const unsigned grid = (unsigned)(total < sms ? total : sms);
-    alignas(64) CUtensorMap tmap;
-    const bool tma = encode_rows_tmap(job, max_rows_per_segment, segments, &tmap);
+    alignas(64) CUtensorMap tmap, tmap2;
+    bool tma = encode_rows_tmap(job, max_rows_per_segment, segments, &tmap);
+    if (two) {
+      HashJob j2 = job;
+      j2.x = job.x2, j2.rows = job.rows2;
+      tma = encode_rows_tmap(j2, j2.rows, 1, &tmap2) && tma;
+    } else {
+      tmap2 = tmap;
+    }
     if (job.w_image != nullptr && (image_built == nullptr || !*image_built)) {  // scratch of kWImageBytes: filled once per call
       build_w_image_kernel<<<(job.d * N + 255) / 256, 256, 0, stream>>>(job.W, job.d, job.b, N,
                                                                        static_cast<unsigned char*>(const_cast<void*>(job.w_image)));
@@ -260,7 +278,7 @@ int launch_hash(const HashJob& job, long long max_rows_per_segment, int segments
       attr[0].val.programmaticStreamSerializationAllowed = 1;
       lc.attrs = attr;
       lc.numAttrs = (pdl && pdl_enabled()) ? 1 : 0;
-      HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, kernel, job, total, tiles, tmap));
+      HE_CUDA_CHECK(cudaLaunchKernelEx(&lc, kernel, job, total, tiles, tmap, tmap2));
       return HE_OK;
     };
     int rc;
@@ -619,17 +637,14 @@ int he_decode_step(const he_config* cfg, const he_cache* cache, const void* q, c
     job.row_stride = cfg->head_dim;
     job.w_image = reinterpret_cast<char*>(cache->step_scratch) +
                   align_up((size_t)units_ll * (cfg->group_size + 1) * Wd * 4, 256);
+    // the query rows and the key rows go through one launch; the key codes follow the query codes in the scratch
     job.x = q;
     job.rows = units_ll * cfg->group_size;
+    job.x2 = k;
+    job.rows2 = units_ll;
     job.out = cache->step_scratch;
     bool image_built = false;
     if (int rc = launch_hash(job, job.rows, 1, st, &image_built)) return rc;
-    job.x = k;
-    job.out = cache->step_scratch + job.rows * Wd;
-    job.rows = units_ll;
-    // the key rows are hashed by a programmatically launched kernel: it needs nothing from the query-row kernel, so
-    // it may run beside it; it ends only after that kernel has ended, which is what the scan kernel's wait relies on
-    if (int rc = launch_hash(job, job.rows, 1, st, &image_built, true)) return rc;
     a.new_codes = cache->step_scratch;
   }
   if (cache->budget_host != nullptr && cfg->batch <= kMaxBudgetVals) {
