@@ -775,10 +775,19 @@ int prefill_impl(int variant /* 0: Algorithm 1, 1: averaged Hamming, 2: L2 norm 
   record_phase(3, st);
   // phase 3: surviving K / V rows into their slots
   GatherArgs ga{*cfg, *cache, k, v, kv_strides[0], kv_strides[1], kv_strides[2], max_prompt_len};
-  const long long per_unit = 2LL * cfg->max_budget * (cfg->head_dim * es / 16);
-  const long long gx = (per_unit + kGatherThreads * kGatherUnroll - 1) / (kGatherThreads * kGatherUnroll);
+  const int cpr = cfg->head_dim * es / 16;
   if (units > 65535) return fail(HE_ERR_UNSUPPORTED, "more than 65535 units in one prefill call");
-  prefill_gather_kernel<<<dim3((unsigned)gx, (unsigned)units), kGatherThreads, 0, st>>>(ga);
+  if (cpr <= kGatherThreads && (cpr & (cpr - 1)) == 0) {  // rows of a power-of-two number of 16-byte chunks
+    int lg = 0;
+    while ((1 << lg) < cpr) ++lg;
+    const int rows_per_cta = (kGatherThreads >> lg) * kGatherRows;
+    const long long gx = ((long long)cfg->max_budget + rows_per_cta - 1) / rows_per_cta;
+    prefill_gather_rows_kernel<<<dim3((unsigned)gx, (unsigned)units), kGatherThreads, 0, st>>>(ga, lg);
+  } else {
+    const long long per_unit = 2LL * cfg->max_budget * cpr;
+    const long long gx = (per_unit + kGatherThreads * kGatherUnroll - 1) / (kGatherThreads * kGatherUnroll);
+    prefill_gather_kernel<<<dim3((unsigned)gx, (unsigned)units), kGatherThreads, 0, st>>>(ga);
+  }
   HE_CUDA_CHECK(cudaGetLastError());
   record_phase(4, st);
   return HE_OK;

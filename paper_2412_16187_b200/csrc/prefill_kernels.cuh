@@ -541,4 +541,50 @@ __global__ void __launch_bounds__(kGatherThreads) prefill_gather_kernel(const Ga
     }
 }
 
+// The same copy for rows of a power-of-two number of 16-byte chunks (every supported head size but the odd ones): a
+// group of `cpr` threads owns a slot at a time, reads its position once and moves the K row and the V row, 16 bytes each
+// per thread; kGatherRows slots per group, so eight loads per thread are in flight. No division anywhere.
+constexpr int kGatherRows = 4;
+__global__ void __launch_bounds__(kGatherThreads) prefill_gather_rows_kernel(const GatherArgs a, int lg_cpr) {
+  const he_config& cfg = a.cfg;
+  const long long unit = blockIdx.y;
+  const int s = (int)(unit / cfg.n_kv_heads), h = (int)(unit % cfg.n_kv_heads);
+  const int es = esize_of(cfg.dtype);
+  const long long Cmax = cfg.max_budget;
+  const int fill = min(max(a.ca.fill[unit], 0), (int)Cmax);
+  const int groups = kGatherThreads >> lg_cpr;
+  const int j0 = blockIdx.x * groups * kGatherRows;
+  if (j0 >= fill) return;
+  const int ch = threadIdx.x & ((1 << lg_cpr) - 1), g = threadIdx.x >> lg_cpr;
+  const int32_t* pp = a.ca.pos + unit * Cmax;
+  const char* kb = static_cast<const char*>(a.k) + (s * a.s0 + h * a.s1) * es;
+  const char* vb = static_cast<const char*>(a.v) + (s * a.s0 + h * a.s1) * es;
+  long long tok[kGatherRows];
+#pragma unroll
+  for (int i = 0; i < kGatherRows; ++i) {
+    const int j = j0 + i * groups + g;
+    tok[i] = -1;
+    if (j < fill) {
+      const long long tk = __ldg(pp + j);
+      if (HE_IN_RANGE(tk, a.Nmax)) tok[i] = tk;  // (a slot of a valid cache names a prompt token)
+    }
+  }
+  uint4 kv[kGatherRows], vv[kGatherRows];
+#pragma unroll
+  for (int i = 0; i < kGatherRows; ++i)
+    if (tok[i] >= 0) {
+      kv[i] = __ldg(reinterpret_cast<const uint4*>(kb + tok[i] * a.s2 * es) + ch);
+      vv[i] = __ldg(reinterpret_cast<const uint4*>(vb + tok[i] * a.s2 * es) + ch);
+    }
+  uint4* kd = reinterpret_cast<uint4*>(a.ca.k_cache) + ((unit * Cmax) << lg_cpr) + ch;
+  uint4* vd = reinterpret_cast<uint4*>(a.ca.v_cache) + ((unit * Cmax) << lg_cpr) + ch;
+#pragma unroll
+  for (int i = 0; i < kGatherRows; ++i)
+    if (tok[i] >= 0) {
+      const long long j = j0 + i * groups + g;
+      kd[j << lg_cpr] = kv[i];
+      vd[j << lg_cpr] = vv[i];
+    }
+}
+
 }  // namespace he
