@@ -58,8 +58,8 @@ struct StepStager {
 // ------------------------------------------------------------------------------------------------ scheduling
 
 // Replay work is very uneven when budgets are ragged (a unit costs about (N - C) * C slot visits) and a CTA
-// runs one unit at a time, so units are dealt to one bin per SM, largest first, each to the currently lightest
-// bin. A replay CTA drains the bin of the SM it runs on and then helps other bins. The result never depends on
+// runs one unit at a time, so units are sorted by work and dealt to one bin per SM, largest first, in a snake over
+// the bins. A replay CTA drains the bin of the SM it runs on and then helps other bins. The result never depends on
 // which CTA runs which unit; only the time does.
 //
 // sched layout (int32): [0] nbins, [1] units, [2 .. 2+nbins] bin_start (nbins + 1 entries),
@@ -132,58 +132,24 @@ __global__ void __launch_bounds__(kSchedThreads) prefill_schedule_kernel(const h
       }
       __syncthreads();
     }
-  if (tid < 32) {  // greedy: next-largest unit to the lightest bin (lowest index on ties)
-    // Bin loads live in registers (lane l owns bins l, l + 32, ...), scaled to 23 bits so that (load << 8 | bin) fits
-    // one word and the lightest bin is a single redux.sync. The scaling only affects balance, never correctness.
-    // The owner lane of the chosen bin also counts the bin's units, so a unit's place inside its bin is known at once.
-    constexpr int kOwn = kMaxBins / 32;
-    unsigned long long total = 0ull;
-    for (int i = tid; i < units; i += 32) total += keys[i] >> 20;
-    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
-    int shift = 0;
-    while ((total >> shift) >= (1ull << 23)) ++shift;
-    uint32_t own[kOwn], cnt[kOwn];
-#pragma unroll
-    for (int k = 0; k < kOwn; ++k) own[k] = 0u, cnt[k] = 0u;
-    unsigned long long key_next = units > 0 ? keys[0] : 0ull;
-    for (int i = 0; i < units; ++i) {
-      const uint32_t wk = (uint32_t)((key_next >> 20) >> shift);
-      if (i + 1 < units) key_next = keys[i + 1];
-      uint32_t best = 0xFFFFFFFFu;
-#pragma unroll
-      for (int k = 0; k < kOwn; ++k) {
-        const int bb = tid + 32 * k;
-        if (bb < nbins) best = min(best, (own[k] << 8) | (uint32_t)bb);
-      }
-      best = __reduce_min_sync(0xFFFFFFFFu, best);
-      const int bb = (int)(best & 0xFFu);
-#pragma unroll
-      for (int k = 0; k < kOwn; ++k)
-        if (bb == tid + 32 * k) {
-          own[k] += wk;
-          bin_of[i] = (unsigned char)bb;
-          pos_of[i] = (unsigned short)cnt[k];
-          cnt[k] += 1u;
-        }
-    }
-    // bin_start: exclusive prefix of the bins' counts (bin = lane + 32 k: prefix over lanes for each k, then over k)
-    uint32_t before_k = 0u;
-#pragma unroll
-    for (int k = 0; k < kOwn; ++k) {
-      uint32_t inc = cnt[k];
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if (tid >= o) inc += v;
-      }
-      const int bb = tid + 32 * k;
-      if (bb < nbins) {
-        start_s[bb] = (int)(before_k + inc - cnt[k]);
-        bin_start[bb] = (int)(before_k + inc - cnt[k]);
-      }
-      before_k += __shfl_sync(0xFFFFFFFFu, inc, 31);
-    }
-    if (tid == 0) bin_start[nbins] = units;
+  // Sorted units are dealt to the bins in a snake (ranks 0 .. nbins-1 forwards, the next nbins backwards, ...): every
+  // bin gets one unit of each round, the heavy bins of one round the light units of the next. A greedy
+  // lightest-bin-first deal balances a little better on paper but is a serial loop over the units (65 us for 512 of
+  // them, 2 % of the call), and the replay CTAs steal from other bins once their own is empty, which evens out what
+  // the deal leaves (measured: the call time does not depend on the cost model at all).
+  const int rounds_full = units / nbins, rem = units - rounds_full * nbins;
+  for (int bb = tid; bb <= nbins; bb += kSchedThreads) {
+    // units in bins below bb: the full rounds give each bin one; the partial round (if any) fills from the front when
+    // its number is even and from the back when it is odd
+    const int extra = (rounds_full & 1) == 0 ? min(bb, rem) : max(0, bb - (nbins - rem));
+    const int st = bb * rounds_full + extra;
+    if (bb < nbins) start_s[bb] = st;
+    bin_start[bb] = st;
+  }
+  for (int i = tid; i < units; i += kSchedThreads) {
+    const int round = i / nbins, k = i - round * nbins;
+    bin_of[i] = (unsigned char)((round & 1) == 0 ? k : nbins - 1 - k);
+    pos_of[i] = (unsigned short)round;
   }
   __syncthreads();
   // sorted order, so each bin lists its largest unit first
