@@ -454,12 +454,12 @@ int launch_replay_reg(const ReplayArgs& a, long long units, cudaStream_t stream)
 
 // Tensor-core replay: one persistent CTA per SM, for budgets up to 12288 slots. Up to 4096 slots the unit's tables sit in
 // shared memory, beyond that they are the cache's own arrays.
-template <int WORDS, bool GLOBAL_TABLE, bool FP8, bool PROT = false>
+template <int WORDS, bool GLOBAL_TABLE, bool FP8, bool PROT = false, bool RUNS = true>
 int launch_replay_tc_one(const ReplayArgs& a0, long long units, cudaStream_t stream) {
   ReplayArgs a = a0;
   a.smem_slots = (a.cfg.max_budget + kRtTile - 1) / kRtTile * kRtTile;
   const size_t smem = rt_layout(WORDS, a.smem_slots, a.cfg.group_size, !GLOBAL_TABLE, FP8).total;
-  if (int rc = set_smem(prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8, PROT>, smem)) return rc;
+  if (int rc = set_smem(prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8, PROT, RUNS>, smem)) return rc;
   int sms = 0;
   if (int rc = sm_count(&sms)) return rc;
   const int nbins = sms < kMaxBins ? sms : kMaxBins;
@@ -467,7 +467,7 @@ int launch_replay_tc_one(const ReplayArgs& a0, long long units, cudaStream_t str
   prefill_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(a.cfg, a.ca.budget, a.prompt_len, nbins, a.sched, 6700);
   HE_CUDA_CHECK(cudaGetLastError());
   const long long grid = units < sms ? units : sms;
-  prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8, PROT><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);
+  prefill_replay_tc_kernel<WORDS, GLOBAL_TABLE, FP8, PROT, RUNS><<<(unsigned)grid, kRtThreads, smem, stream>>>(a);
   HE_CUDA_CHECK(cudaGetLastError());
   return HE_OK;
 }
@@ -483,7 +483,12 @@ int launch_replay_tc(const ReplayArgs& a, long long units, cudaStream_t stream) 
   if (a.cfg.n_sink > 0 || a.cfg.n_recent > 0)  // protected windows
     return fp8 ? launch_replay_tc_one<WORDS, GLOBAL_TABLE, true, true>(a, units, stream)
                : launch_replay_tc_one<WORDS, GLOBAL_TABLE, false, true>(a, units, stream);
-  if (fp8) return launch_replay_tc_one<WORDS, GLOBAL_TABLE, true>(a, units, stream);
+  if (fp8) {
+    // no unit of such a launch can use the run-based resolver loop (every table keeps its tiles' second-largest keys)
+    if (!GLOBAL_TABLE && a.cfg.max_budget <= kRtSecondMaxTiles * kRtTile)
+      return launch_replay_tc_one<WORDS, false, true, false, false>(a, units, stream);
+    return launch_replay_tc_one<WORDS, GLOBAL_TABLE, true>(a, units, stream);
+  }
   return launch_replay_tc_one<WORDS, GLOBAL_TABLE, false>(a, units, stream);
 }
 

@@ -46,6 +46,7 @@ constexpr int kRtMaxSlotsGlobal = 12288;  // largest budget at all: the tables t
 constexpr int kRtKeyShift = 14;
 constexpr int kRtIdxMask = (1 << kRtKeyShift) - 1;
 constexpr int kRtStaleLimit = 64;  // repairs after which a block is cut short
+constexpr int kRtSecondMaxTiles = 8;  // tables up to this many tiles also keep each tile's second-largest key (8-bit operands)
 constexpr int kRtFastNum = 3, kRtFastDen = 10;  // run-based resolver while fewer than NUM / DEN of a unit's steps are not easy
 constexpr int kRtAtomBytes = kRtRows * 128;  // one 64-column K-major swizzle atom of a 128-row operand tile
 
@@ -145,8 +146,11 @@ __device__ __forceinline__ int rt_dist(const uint32_t* h, const uint32_t* q, int
 // operands. The resolver treats a best base slot that is not eligible at this step like a stale one (the repair
 // then takes the tile's best eligible slot), and a token that enters at step r joins the new entries only at step
 // r + n_recent + 1, when it stops being recent; until then, and in the next block, it cannot win.
-template <int WORDS, bool GLOBAL_TABLE, bool FP8, bool PROT = false>
+// RUNS = false leaves the run-based resolver loop out of the kernel: for launches none of whose units can use it (see
+// `second` below) the sequential loop alone compiles to tighter code (5 % of the call at 1024-slot budgets).
+template <int WORDS, bool GLOBAL_TABLE, bool FP8, bool PROT = false, bool RUNS = true>
 __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const ReplayArgs a) {
+  constexpr bool kRuns = RUNS && !PROT;
   constexpr int ATOMS = (WORDS == 2 && !FP8) ? 2 : 1;
   constexpr int KB = 32 * WORDS;             // code columns of the contraction
   constexpr int KSTEPS = FP8 ? KB / 32 + 1 : (KB + 16) / 16;  // MMA instructions per tile (the last one holds the key columns)
@@ -163,7 +167,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   __shared__ __align__(8) unsigned long long bars[4 * NSTAGE + 1];  // the last one: drain barrier of the abort path
   __shared__ uint32_t tmem_base_s;
   __shared__ volatile int abort_flag;
-  __shared__ int s_unit, s_done, s_fast;
+  __shared__ int s_unit, s_done, s_fast, s_hold, s_backoff;
   __shared__ uint16_t entry_slot[PROT ? kRtRows : 1];  // PROT: the slot each of the block's steps wrote to
   // four code bits -> four bf16 values: operand B takes +-1 (bit set: +1), operand A -+2^13 (bit set: -2^13)
   __shared__ uint2 s_lut_a[16], s_lut_b[16];
@@ -186,7 +190,6 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
   int16_t* owner = reinterpret_cast<int16_t*>(smem + L.owner);
   int32_t* Mx = reinterpret_cast<int32_t*>(smem + L.m);
   constexpr bool SECOND = FP8 && !GLOBAL_TABLE;  // the readers may also keep each tile's second-largest key
-  constexpr int kSecondMaxTiles = 8;  // ... for small tables only: see `second` below
   int32_t* Mx2 = reinterpret_cast<int32_t*>(smem + L.m2);
   int32_t* RB = reinterpret_cast<int32_t*>(smem + L.rb);
   int32_t* UB = reinterpret_cast<int32_t*>(smem + L.ub);  // per step: no new entry's key can exceed this
@@ -263,7 +266,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     // the readers five instructions per two elements instead of one. Measured on B200: with 1024 slots (8 tiles, a
     // fifth of the steps stale) the call gets 8 % faster, with 2048 slots and more the longer tile phase costs more
     // than the repairs saved.
-    const bool second = SECOND && nbase <= kSecondMaxTiles;
+    const bool second = SECOND && nbase <= kRtSecondMaxTiles;
     uint32_t* codes_t = GLOBAL_TABLE ? a.ca.codes + unit * Cmax * WORDS : reinterpret_cast<uint32_t*>(smem + L.codes);
     int32_t* pos_t = GLOBAL_TABLE ? a.ca.pos + unit * Cmax : reinterpret_cast<int32_t*>(smem + L.pos);
     // the first C tokens fill the cache in order; everything beyond `fill` is reset
@@ -275,7 +278,11 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
     // PROT with the tables in global memory: positions are too far away for the resolver's step-ahead checks, so warp 0
     // keeps the slots of the 32 newest tokens in a register ring (lane l: the newest token congruent to l mod 32; the
     // first C tokens sit in slot = position) and sinks are recognised by their slot (they never leave slots 0..n_sink-1).
-    if (tid == 0) s_fast = PROT ? 0 : 1;  // a unit's first block tries the run-based loop
+    if (tid == 0) {
+      s_fast = 0;  // a unit's first block runs the sequential loop and counts
+      s_hold = 0;
+      s_backoff = 2;
+    }
     int myring = -1;
     if (PROT && GLOBAL_TABLE) {
       const int pl = fill0 - 1 - ((fill0 - 1 - lane) & 31);
@@ -568,7 +575,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
               uint32_t v[32];
               tc_ld32(taddr + c * 32, v);
               tc_wait_ld();
-              if (s_fast) {
+              if (kRuns && s_fast) {
 #pragma unroll
                 for (int k = 0; k < 32; ++k)
                   if (c * 32 + k < tid) dmax = fmaxf(dmax, __uint_as_float(v[k]));
@@ -596,8 +603,8 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
           for (int i = 0; i < nbase; ++i) rb = max(rb, Mx[tid * mp + i]);
           RB[tid] = rb;
         }
-        if (s_fast) asm volatile("bar.sync 2, 128;" ::: "memory");  // the four reader warps: RB and UB are complete
-        if (ok && s_fast) {
+        if (kRuns && s_fast) asm volatile("bar.sync 2, 128;" ::: "memory");  // the four reader warps: RB and UB are complete
+        if (kRuns && ok && s_fast) {
           // what the resolver's easy-run test needs of step `tid`, in one word: the slot of its best base key (14 bits),
           // whether a new entry might beat that key (bit 14), and how many steps back the nearest earlier step with the
           // same slot lies (bits 16-20; 0: none among the 31 steps before it)
@@ -655,14 +662,16 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
         // of them is settled by the warp's lanes side by side. Only the other steps - a stale maximum, a new entry that
         // may win, the scoring pass - go through the sequential path below, one at a time.
         // The run test costs about as much as a sequential step and fails at every step that is not easy, so it only
-        // pays while those are few (measured break-even: three steps in ten). Each block counts the steps that were not
-        // easy, whichever loop it ran, and the unit's next block picks its loop by that count; s_fast also tells the
-        // readers whether the next block needs the run test's tables (UB, PS) at all.
-        const bool FAST = !PROT && s_fast != 0;
+        // pays while those are few (measured break-even: three steps in ten). A unit starts in the sequential loop, which
+        // counts the steps it can tell were not easy; a run-based block counts them exactly, and the unit's next block
+        // picks its loop by that count (a run-based block that did not pay holds the unit in the sequential loop for a
+        // growing number of blocks). s_fast also tells the readers whether the next block needs the run test's tables
+        // (UB, PS) at all.
+        const bool FAST = kRuns && s_fast != 0;
         int n_not_easy = 0;
-        // the loop is compiled twice, so that the plain sequential form keeps the tight code it had before the run test
-        auto resolve_block = [&](auto fast_c) {
-          constexpr bool FASTC = decltype(fast_c)::value;
+        // the loop is compiled in separate forms, so that the plain sequential one keeps the tight code it had before the run test
+        auto resolve_block = [&](auto fast_c, auto count_c) {
+          constexpr bool FASTC = decltype(fast_c)::value, COUNT = decltype(count_c)::value;
           bool resume = false;  // re-entering the sequential path at the same step after a repair or the scoring pass
           bool vb_dirty = false;
           if (FASTC) {  // no entry of this block is resident yet
@@ -739,7 +748,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
               const int k2 = (int)((dd.y & 0xFFFFu) << kRtKeyShift) + vb2;
               const int k3 = (int)((dd.y >> 16) << kRtKeyShift) + vb3;
               const int kn = __reduce_max_sync(0xFFFFFFFFu, max(max(k0, k1), max(k2, k3)));
-              if (!PROT && !FASTC) n_not_easy += (own_kb >= 0 || kn >= kb) ? 1 : 0;  // (a repaired step re-enters and counts twice)
+              if (COUNT && !FASTC) n_not_easy += (own_kb >= 0 || kn >= kb) ? 1 : 0;  // (a repaired step re-enters and counts twice)
               // best base slot: the tile maxima are upper bounds; one that points at an evicted slot needs a repair
               if (kb > kn && own_kb >= 0) {
                 status = 1;
@@ -886,11 +895,35 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             }
           }
         };
-        if (FAST) resolve_block(std::true_type{}); else resolve_block(std::false_type{});
+        // the sequential loop counts only when its count can matter: two or three instructions more per step cost it 5 %
+        const bool counting = kRuns && !second && s_hold == 0;
+        if (FAST) resolve_block(std::true_type{}, std::true_type{});
+        else if (counting) resolve_block(std::false_type{}, std::true_type{});
+        else resolve_block(std::false_type{}, std::false_type{});
         if (lane == 0) {
           s_done = done;
           // (the sequential loop sees only part of what makes a step not easy, hence its stricter bar for switching back)
-          s_fast = !PROT && (FAST ? n_not_easy * kRtFastDen < done * kRtFastNum : n_not_easy * 10 < done);
+          // A run-based block that did not pay sends the unit back to the sequential loop for a number of blocks that
+          // doubles with every failure: the sequential loop's own count misses part of what makes a step not easy, so
+          // without the hold a unit near the bar would try the run test again every other block.
+          bool fast_next;
+          if (FAST) {
+            fast_next = n_not_easy * kRtFastDen < done * kRtFastNum;
+            if (!fast_next) {
+              s_backoff = min(4 * s_backoff, 64);
+              s_hold = s_backoff;
+            } else {
+              s_backoff = 2;
+            }
+          } else if (!counting) {
+            if (s_hold > 0) --s_hold;
+            fast_next = false;
+          } else {
+            fast_next = n_not_easy * 10 < done;
+          }
+          // (with the tiles' second-largest keys at hand the sequential loop settles most stale maxima at once and the run
+          // test does not pay: 2.09 against 2.20 ms per call with 1024-slot budgets)
+          s_fast = kRuns && !second && fast_next;
         }
       } else if (tn < N) {
         const int nrows = (N - tn) < kRtRows ? (N - tn) : kRtRows;
