@@ -897,10 +897,11 @@ __global__ void __launch_bounds__(kRtThreads, 1) prefill_replay_tc_kernel(const 
             }
           }
         };
-        // the sequential loop counts only when its count can matter: two or three instructions more per step cost it 5 %
+        // The kernel with the run-based loop holds one sequential form, which always counts (the count is ignored while
+        // the unit is held); a third copy of the loop without the count made the call slower, not faster (code size).
         const bool counting = kRuns && !second && s_hold == 0;
         if (FAST) resolve_block(std::true_type{}, std::true_type{});
-        else if (counting) resolve_block(std::false_type{}, std::true_type{});
+        else if (kRuns) resolve_block(std::false_type{}, std::true_type{});
         else resolve_block(std::false_type{}, std::false_type{});
         if (lane == 0) {
           s_done = done;
