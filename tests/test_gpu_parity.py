@@ -309,10 +309,15 @@ def test_no_kernel_gave_up_on_a_bounded_wait():
     assert device_error_count() == 0
 
 
-def test_large_batch_decode_hashes_new_rows_in_bulk():
-    """4096 units x (G + 1) = 20480 new rows per step: he_decode_step hashes them with the bulk projection kernels
-    into the step scratch and the per-unit kernel only scans. Results must not depend on that choice."""
-    w = wl.CONFIGS["throughput_batch"].scaled(batch=512, budget_lo=40, budget_hi=64, prompt_factor=1, decode_steps=5)
+@pytest.mark.parametrize("batch,dtype", [(512, "bf16"), (515, "bf16"), (512, "f32")],
+                         ids=["whole_tiles", "ragged_tiles", "fp32_cuda_cores"])
+def test_large_batch_decode_hashes_new_rows_in_bulk(batch, dtype):
+    """About 4100 units x (G + 1) = 20500 new rows per step: he_decode_step hashes them with the bulk projection kernels
+    into the step scratch and the per-unit kernel only scans. Results must not depend on that choice. bf16 rows go
+    through ONE launch of the tensor-core kernel as two row ranges (query rows, key rows), here also with row counts
+    that end inside a 128-row tile; fp32 rows go through the CUDA-core kernel, one launch per range."""
+    w = wl.CONFIGS["throughput_batch"].scaled(batch=batch, budget_lo=40, budget_hi=64, prompt_factor=1, decode_steps=5,
+                                               dtype=dtype)
     case = Case(w)
     case.prefill()
     case.compare_state()
