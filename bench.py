@@ -504,14 +504,17 @@ def run_ours(args, w):
             hblock[i, oq:oq + qb] = gq[i].contiguous().view(torch.uint8).flatten().cpu()
             hblock[i, ok_:ok_ + kb] = gk[i].contiguous().view(torch.uint8).flatten().cpu()
             hblock[i, ov:ov + kb] = gv[i].contiguous().view(torch.uint8).flatten().cpu()
-        # The layer replicas' calls of a step are independent, so they alternate between two streams (each with its
-        # own staging): the copies of one overlap the kernel of the other. Every step ends with a synchronise, after
+        # The layer replicas' calls of a step are independent, so they alternate between a few streams (each with its
+        # own staging): the copies of one overlap the kernels and the copies of the others. A 0.79 MB host-to-device copy
+        # costs 38 us back to back on one stream (20 GB/s; the link reaches 54 GB/s only from 16 MB per copy), so several
+        # must be in flight: 1 / 2 / 4 / 8 streams gave 47 / 32 / 29 / 26 us per call. Every step ends with a synchronise, after
         # which that step's victims are readable on the host.
         hvic = torch.empty((R, B, H), dtype=torch.int32).pin_memory()
-        e_streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        e_streams = [torch.cuda.Stream() for _ in range(max(1, min(args.e2e_streams, R)))]
+        ns = len(e_streams)
         stagings = [torch.empty(decode_staging_bytes(caches[0].cfg), dtype=torch.uint8, device="cuda") for _ in e_streams]
         base = hblock.data_ptr()
-        calls = [(c, hvic[r].data_ptr(), stagings[r & 1].data_ptr(), stagings[r & 1].numel(), e_streams[r & 1].cuda_stream)
+        calls = [(c, hvic[r].data_ptr(), stagings[r % ns].data_ptr(), stagings[r % ns].numel(), e_streams[r % ns].cuda_stream)
                  for r, c in enumerate(caches)]
 
         def e2e_step(i):
@@ -531,7 +534,7 @@ def run_ours(args, w):
         t_e2e = time.perf_counter() - t0
         line["e2e"] = {"value": units * n_e2e * R * world / t_e2e, "unit": UNIT, "h2d_bytes_per_step": qb + 2 * kb,
                        "d2h_bytes_per_step": hvic[0].numel() * 4, "us_per_call": 1e6 * t_e2e / (n_e2e * R),
-                       "what": f"he_decode_step_host_block_enqueue, {n_e2e} decode steps x {R} layer replicas on two alternating streams, "
+                       "what": f"he_decode_step_host_block_enqueue, {n_e2e} decode steps x {R} layer replicas on {ns} alternating streams, "
                                "one synchronise and one host read of the victims per step; every call copies its pinned host "
                                "q/k/v block in (one copy) and its victims out inside the timed region"}
 
@@ -725,6 +728,7 @@ def main():
     ap.add_argument("--skip-attend", action="store_true", help="skip the he_attend figure")
     ap.add_argument("--skip-folded", action="store_true", help="skip the secondary all-replicas-in-one-call decode figure")
     ap.add_argument("--e2e-steps", type=int, default=64)
+    ap.add_argument("--e2e-streams", type=int, default=8, help="streams the layer replicas' end-to-end calls alternate between")
     ap.add_argument("--ref-seqs", type=int, default=12, help="sequences in the oracle's bounded sample")
     ap.add_argument("--ref-decode-steps", type=int, default=128)
     args = ap.parse_args()
