@@ -363,27 +363,54 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   const long long n_sched = nseq_dense > 0 ? (long long)s_pref[nseq_dense] : total_tiles;  // tile numbers this grid walks
   int cursor = 0;  // this thread's sequence cursor of the dense schedule
 
+  // Flat rows and the dense schedule number real tiles only, so every role walks t = blockIdx.x, + gridDim.x, ... and all
+  // of them are tiles. There the producer warp and the epilogue warps work out the tiles' coordinates 32 at a time, a
+  // lane per tile, and hand them round by shuffle: done by one thread per tile, that index arithmetic (a search, a
+  // division, 64-bit products) was the longest dependent chain of the kernel's per-tile work.
+  const bool batched = nseq_dense > 0 || job.mode == 0;
   if (warp == 4 && TMA) {
-    // ------------------------------------------------------------------ producer (TMA, one thread)
-    if (lane == 0) {
-      int it = 0;
+    // ------------------------------------------------------------------ producer (TMA, one thread issues)
+    int it = 0;
+    auto issue = [&](int row0, int c2, int c3, int second) -> bool {  // lane 0
+      const int s = it % kTcStages;
+      if (!mbar_wait(empty_bar(s), ((it / kTcStages) & 1) ^ 1, &abort_flag)) return false;
+      mbar_arrive_expect_tx(full_bar(s), (uint32_t)a_stage_bytes);
+      // rows past the tensor's extent are filled with zeros by the copy engine; their codes are not stored
+      for (int kh = 0; kh < KH; ++kh)
+        tma_load_4d(smem_u32(As + s * a_stage_bytes + kh * a_half_bytes), second ? &tmap2 : &tmap, kh * 64, row0, c2, c3, full_bar(s));
+      return true;
+    };
+    if (batched) {
+      bool alive = true;
+      for (long long tb = blockIdx.x; tb < n_sched && alive; tb += 32LL * gridDim.x) {
+        const long long t = tb + (long long)lane * gridDim.x;
+        int row0 = 0, c2 = 0, c3 = 0, second = 0;
+        TcTile tl;
+        if (t < n_sched && tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor))
+          row0 = (int)tl.row0, c2 = tl.c2, c3 = tl.c3, second = tl.second;
+        const long long left = (n_sched - tb + gridDim.x - 1) / gridDim.x;
+        const int cnt = left < 32 ? (int)left : 32;
+        for (int j = 0; j < cnt && alive; ++j) {
+          const int r0 = __shfl_sync(0xFFFFFFFFu, row0, j), a2 = __shfl_sync(0xFFFFFFFFu, c2, j);
+          const int a3 = __shfl_sync(0xFFFFFFFFu, c3, j), sc = __shfl_sync(0xFFFFFFFFu, second, j);
+          int ok = 1;
+          if (lane == 0) ok = issue(r0, a2, a3, sc) ? 1 : 0;
+          alive = __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+          if (alive) ++it;
+        }
+      }
+    } else if (lane == 0) {
       for (long long t = blockIdx.x; t < n_sched; t += gridDim.x) {
         TcTile tl;
         if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor)) continue;
-        const int s = it % kTcStages;
-        if (!mbar_wait(empty_bar(s), ((it / kTcStages) & 1) ^ 1, &abort_flag)) break;
-        mbar_arrive_expect_tx(full_bar(s), (uint32_t)a_stage_bytes);
-        // rows past the tensor's extent are filled with zeros by the copy engine; their codes are not stored
-        for (int kh = 0; kh < KH; ++kh)
-          tma_load_4d(smem_u32(As + s * a_stage_bytes + kh * a_half_bytes), tl.second ? &tmap2 : &tmap, kh * 64, (int)tl.row0, tl.c2,
-                      tl.c3, full_bar(s));
+        if (!issue((int)tl.row0, tl.c2, tl.c3, tl.second)) break;
         ++it;
       }
-      // A CTA that gives up must not hand its shared memory back while a tile copy into it is still under way: wait
-      // (bounded) for the copies of the stages armed last.
-      if (abort_flag)
-        for (int u = it > kTcStages ? it - kTcStages : 0; u < it; ++u) mbar_drain(full_bar(u % kTcStages), (u / kTcStages) & 1);
     }
+    // A CTA that gives up must not hand its shared memory back while a tile copy into it is still under way: wait
+    // (bounded) for the copies of the stages armed last.
+    if (lane == 0 && abort_flag)
+      for (int u = it > kTcStages ? it - kTcStages : 0; u < it; ++u) mbar_drain(full_bar(u % kTcStages), (u / kTcStages) & 1);
   } else if (warp == 4) {
     // ------------------------------------------------------------------ producer (cp.async fallback)
     int it = 0;                // tiles this CTA has started
@@ -463,11 +490,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-3, one row per thread)
     int it = 0;
-    for (long long t = blockIdx.x; t < n_sched; t += gridDim.x) {
-      TcTile tl;
-      if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor)) continue;
+    // one tile: `obase` = index of its first row's first code word in job.out, `ostride` words between rows
+    auto epi_tile = [&](long long obase, int ostride, int nrows) -> bool {
       const int acc = it & 1;
-      if (!__all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(acc), (it >> 1) & 1, &abort_flag))) break;  // warp-uniform
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar(acc), (it >> 1) & 1, &abort_flag))) return false;  // warp-uniform
       tc_fence_after();
       uint32_t code[WORDS];
 #pragma unroll
@@ -490,12 +516,38 @@ __global__ void __launch_bounds__(kTcThreads, 1) hash_rows_tc_kernel(const HashJ
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
       const int r = warp * 32 + lane;
-      if (r < tl.nrows) {
-        uint32_t* o = job.out + tl.out_base + (tl.row0 + r) * tl.out_stride;
+      if (r < nrows) {
+        uint32_t* o = job.out + obase + (long long)r * ostride;
 #pragma unroll
         for (int w = 0; w < WORDS; ++w) o[w] = code[w];
       }
-      ++it;
+      return true;
+    };
+    if (batched) {
+      bool alive = true;
+      for (long long tb = blockIdx.x; tb < n_sched && alive; tb += 32LL * gridDim.x) {
+        const long long t = tb + (long long)lane * gridDim.x;
+        long long ob = 0;
+        int os = 0, nr = 0;  // (a tile that turned out empty would still be consumed, and store nothing)
+        TcTile tl;
+        if (t < n_sched && tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor))
+          ob = tl.out_base + tl.row0 * tl.out_stride, os = (int)tl.out_stride, nr = tl.nrows;
+        const long long left = (n_sched - tb + gridDim.x - 1) / gridDim.x;
+        const int cnt = left < 32 ? (int)left : 32;
+        for (int j = 0; j < cnt && alive; ++j) {
+          const long long obj = __shfl_sync(0xFFFFFFFFu, ob, j);
+          const int osj = __shfl_sync(0xFFFFFFFFu, os, j), nrj = __shfl_sync(0xFFFFFFFFu, nr, j);
+          alive = epi_tile(obj, osj, nrj);
+          if (alive) ++it;
+        }
+      }
+    } else {
+      for (long long t = blockIdx.x; t < n_sched; t += gridDim.x) {
+        TcTile tl;
+        if (!tc_tile<WORDS>(job, t, tiles_per_seg, &tl, s_len, s_bud, s_pref, nseq_dense, &cursor)) continue;
+        if (!epi_tile(tl.out_base + tl.row0 * tl.out_stride, (int)tl.out_stride, tl.nrows)) break;
+        ++it;
+      }
     }
   }
 
